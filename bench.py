@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the PaFu-KV inference hot path (score -> select -> compact -> chunk attention).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One "step" is one pass of the whole path over one layer's synthetic inputs.  The default
+workload is the single Wan-1.3B-class layer: 12 heads x 128, a 28 080-token cache pruned to
+14 040 (1560 sink + 4680 recent + 7800 by salience), 4680 chunk queries.  Prints one JSON line.
+
+`value` is chunk-attention TFLOP/s over the whole step (attention FLOPs / step time, all four
+kernels included) with inputs resident in HBM; `roofline` describes the attention kernel alone;
+`e2e` is the same metric through pafu_step_host with pinned host buffers; `cpu_baseline` is the
+CPU oracle timed on a bounded sample.  `--impl reference` times that oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "chunk-attn TFLOP/s over salience-pruned KV; ms/denoise step; % of roofline"
+UNIT = "TFLOP/s"
+N_LAYERS_PER_DENOISE_STEP = 30
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.05)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        inside = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.05] or [l for (_, l) in self.lines[-3:]]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in inside:
+            f = [x.strip() for x in l.split(",")]
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def pick_workload(name: str):
+    from paper_2601_21896_b200 import workloads as wl
+    if name in ("wan1.3b_layer", "default"):
+        return wl.wan13b_layer()
+    if name.startswith("wan1.3b_layer_b"):
+        return wl.wan13b_layer(int(name.rsplit("b", 1)[1]) / 100.0)
+    return wl.CONFIGS[name]()
+
+
+def algorithmic_work(w):
+    """Bytes / flops the method itself must move or compute per step (per layer)."""
+    dm = w.d_model
+    nT, nB, nQ = sum(w.T), int(w.cu("B")[-1]), sum(w.Lq)
+    return {
+        "score_bytes": nT * dm * 2 + nT * 4,
+        "score_flops": 2 * nT * dm * w.d_hidden,
+        "select_bytes": nT * 4 + nB * 4,
+        "compact_bytes": 2 * (2 * nB * dm * 2) + nB * 4,
+        "attn_flops": w.attn_flops(),
+        "attn_bytes": (2 * nQ + 2 * nB + 2 * nQ) * dm * 2,
+    }
+
+
+# ------------------------------------------------------------------------------------ oracle
+def oracle_sampled_step(w, d, n_score_tokens, n_rows, seed=0):
+    """One bounded-sample pass of the oracle; returns the per-part seconds and the estimate of
+    the full step (score and attention scaled by the fraction of tokens / query rows done)."""
+    import oracle
+    from paper_2601_21896_b200 import workloads as wl
+    cuT, cuQ = w.cu("T"), w.cu("Lq")
+    nT = int(cuT[-1])
+    t0 = time.perf_counter()
+    tok = min(n_score_tokens, nT)
+    oracle.score(d["K"].reshape(nT, -1)[:tok], d["w1"], d["b1"], d["w2"], d["b2"], w.act, w.final)
+    t_score = time.perf_counter() - t0
+    scores = wl.random_scores(nT, seed=seed, kind="normal")   # stand-in scores for the rest of the path
+    t0 = time.perf_counter()
+    idx = [oracle.select(scores[cuT[s]:cuT[s + 1]], w.n_sink, w.n_recent, w.budget[s])
+           for s in range(w.n_streams)]
+    t_select = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    Kc = [oracle.compact(d["K"][cuT[s]:cuT[s + 1]], idx[s]) for s in range(w.n_streams)]
+    Vc = [oracle.compact(d["V"][cuT[s]:cuT[s + 1]], idx[s]) for s in range(w.n_streams)]
+    t_compact = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    rows_done = 0
+    for s in range(w.n_streams):
+        rows = wl.sample_rows(w.Lq[s], max(1, n_rows // w.n_streams), seed=seed, tag=s)
+        rows = rows[: max(1, n_rows // w.n_streams)]
+        oracle.attention(d["Q"][cuQ[s]:cuQ[s + 1]], Kc[s], Vc[s], d["Kq"][cuQ[s]:cuQ[s + 1]],
+                         d["Vq"][cuQ[s]:cuQ[s + 1]], rows=rows)
+        rows_done += len(rows)
+    t_attn = time.perf_counter() - t0
+    est = t_score * nT / tok + t_select + t_compact + t_attn * sum(w.Lq) / rows_done
+    return {"score_s": t_score, "select_s": t_select, "compact_s": t_compact, "attn_s": t_attn,
+            "score_tokens": tok, "attn_rows": rows_done, "full_step_est_s": est,
+            "spent_s": t_score + t_select + t_compact + t_attn}
+
+
+def cpu_baseline(w, d, budget_s=15.0):
+    import oracle
+    probe = oracle_sampled_step(w, d, 64, 1 * w.n_streams)
+    per_tok = probe["score_s"] / probe["score_tokens"]
+    per_row = probe["attn_s"] / probe["attn_rows"]
+    n_tok = int(max(64, min(sum(w.T), 0.3 * budget_s / max(per_tok, 1e-9))))
+    n_rows = int(max(w.n_streams, min(sum(w.Lq), 0.6 * budget_s / max(per_row, 1e-9))))
+    r = oracle_sampled_step(w, d, n_tok, n_rows)
+    return {"value": w.attn_flops() / r["full_step_est_s"] / 1e12, "unit": UNIT,
+            "cores": oracle.n_threads(), "kind": "oracle",
+            "sample": "score on %d of %d tokens, select and compact in full, attention on %d of %d "
+                      "query rows (all heads); %.1f s of CPU work, step time extrapolated to the full "
+                      "workload (%.1f s)" % (r["score_tokens"], sum(w.T), r["attn_rows"], sum(w.Lq),
+                                             r["spent_s"], r["full_step_est_s"])}
+
+
+def run_reference(args):
+    """The reference arm is the CPU oracle as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2601_21896_b200 import workloads as wl
+    w = pick_workload(args.workload)
+    steps = args.steps if args.steps is not None else 3
+    warmup = args.warmup if args.warmup is not None else 1
+    d = wl.make_layer(w)
+    probe = oracle_sampled_step(w, d, 64, w.n_streams)
+    per_step_budget = max(0.2, 90.0 / (steps + warmup))
+    n_tok = int(max(16, min(sum(w.T), 0.3 * per_step_budget / (probe["score_s"] / probe["score_tokens"]))))
+    n_rows = int(max(w.n_streams, min(sum(w.Lq), 0.6 * per_step_budget / (probe["attn_s"] / probe["attn_rows"]))))
+    for _ in range(warmup):
+        oracle_sampled_step(w, d, n_tok, n_rows)
+    est = []
+    for _ in range(steps):
+        est.append(oracle_sampled_step(w, d, n_tok, n_rows)["full_step_est_s"])
+    ms = 1e3 * float(np.mean(est))
+    value = w.attn_flops() / (ms * 1e-3) / 1e12
+    sample = ("each step: score on %d of %d tokens, select and compact in full, attention on %d of %d "
+              "query rows; step time extrapolated to the full workload" % (n_tok, sum(w.T), n_rows, sum(w.Lq)))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "heads": w.n_heads, "d_head": w.d_head, "cache_tokens": list(w.T),
+                       "budget": list(w.budget), "chunk_tokens": list(w.Lq)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# -------------------------------------------------------------------------------------- ours
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2601_21896_b200 as pafu
+    from paper_2601_21896_b200 import workloads as wl
+    from paper_2601_21896_b200.harness import Layer
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the CUDA path has no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    steps = args.steps if args.steps is not None else 200
+    warmup = max(3, args.warmup if args.warmup is not None else 10)
+    w = pick_workload(args.workload)
+    work = algorithmic_work(w)
+    peaks = measured_peaks()
+
+    # independent layer units per rank (weak scaling: no data-path collective)
+    n_sets = args.sets
+    layers, host0 = [], None
+    for i in range(n_sets):
+        d = wl.make_layer(w, seed=0, layer=rank * n_sets + i)
+        if i == 0:
+            host0 = d
+        layers.append(Layer(w, d, want_lse=False, want_slc=True))
+    stream = torch.cuda.current_stream()
+
+    def new_events(n):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in ev:
+            e.record(stream)          # torch creates the cudaEvent_t on first record
+        return ev
+
+    for i in range(warmup):
+        layers[i % n_sets].step()
+    for L in layers:
+        L.check_status()
+    step_events = [new_events(5) for _ in range(steps)]
+    handles = [pafu.event_handles(ev) for ev in step_events]
+    start, end = new_events(2)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.15)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    start.record(stream)
+    for i in range(steps):
+        pafu.pafu_step_timed(layers[i % n_sets].args, handles[i])
+    end.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    for L in layers:
+        L.check_status()
+    total_ms = start.elapsed_time(end)
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    parts = np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(4)] for ev in step_events])
+    k_ms = parts.mean(axis=0)          # score, select, compact, attn
+    ms_per_step = total_ms / steps
+    value = world * work["attn_flops"] / (ms_per_step * 1e-3) / 1e12
+
+    # ---- e2e: host buffers through pafu_step_host (H2D of inputs + D2H of results timed)
+    L0 = layers[0]
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+    hin = {k: pin(v) for k, v in host0.items()}
+    h_scores = torch.empty(L0.nT, dtype=torch.float32).pin_memory()
+    h_idx = torch.empty(L0.nB, dtype=torch.int32).pin_memory()
+    h_O = torch.empty((L0.nQ, w.n_heads, w.d_head), dtype=torch.int16).pin_memory()
+    hhead = pafu.Head(hin["w1"], hin["b1"], hin["w2"], hin["b2"], w.act, w.final)
+    arena = torch.empty(pafu.pafu_step_host_arena_bytes(L0.shape, L0.policy, hhead), dtype=torch.uint8, device="cuda")
+    hargs = pafu.step_args(L0.shape, hhead, L0.policy, hin["K"], hin["V"], hin["Q"], hin["Kq"], hin["Vq"], 0.0,
+                           h_scores, h_idx, None, None, None, h_O, None, None)
+    e2e_steps = max(3, min(steps, 10))
+    for _ in range(2):
+        pafu.pafu_step_host(hargs, arena)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e0, e1 = new_events(2)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        pafu.pafu_step_host(hargs, arena)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(int(v.numel() * v.element_size()) for v in hin.values())
+    d2h = int(h_scores.numel() * 4 + h_idx.numel() * 4 + h_O.numel() * 2)
+    e2e_value = world * work["attn_flops"] / (e2e_ms * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    burst = total_ms < 1500.0
+    peak_tf = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+    attn_tf = work["attn_flops"] / (k_ms[3] * 1e-3) / 1e12
+    gbs = lambda b, ms: b / (ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "heads": w.n_heads, "d_head": w.d_head, "cache_tokens": list(w.T),
+                   "budget": list(w.budget), "n_sink": w.n_sink, "n_recent": w.n_recent,
+                   "chunk_tokens": list(w.Lq), "head_mlp": [w.d_model, w.d_hidden, w.d_out],
+                   "l2": "inputs larger than L2: %d independent layer buffer sets (>= 300 MB each) used "
+                         "round-robin, no flush" % n_sets},
+        "roofline": {"kernel": "chunk attention", "bound": "tensor", "achieved": attn_tf, "peak": peak_tf,
+                     "unit": "TFLOP/s", "frac": attn_tf / peak_tf, "traffic": None,
+                     "peak_source": "%s, %s" % (peaks["source"], "burst" if burst else "sustained")},
+        "kernels": {
+            "score": {"ms": k_ms[0], "GB/s": gbs(work["score_bytes"], k_ms[0]),
+                      "TFLOP/s": work["score_flops"] / (k_ms[0] * 1e-3) / 1e12,
+                      "hbm_frac": gbs(work["score_bytes"], k_ms[0]) / peaks["hbm_gbs"]},
+            "select": {"ms": k_ms[1], "GB/s": gbs(work["select_bytes"], k_ms[1])},
+            "compact": {"ms": k_ms[2], "GB/s": gbs(work["compact_bytes"], k_ms[2]),
+                        "hbm_frac": gbs(work["compact_bytes"], k_ms[2]) / peaks["hbm_gbs"]},
+            "attn": {"ms": k_ms[3], "TFLOP/s": attn_tf, "tensor_frac": attn_tf / peak_tf},
+            "score+select+compact": {
+                "ms": float(k_ms[:3].sum()),
+                "GB/s": gbs(work["score_bytes"] + work["select_bytes"] + work["compact_bytes"], k_ms[:3].sum()),
+                "hbm_frac": gbs(work["score_bytes"] + work["select_bytes"] + work["compact_bytes"],
+                                k_ms[:3].sum()) / peaks["hbm_gbs"]},
+        },
+        "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step,
+        "peaks": peaks,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "api": "pafu_step_host (pinned host buffers)"},
+        "gpu_launches": 4 * steps,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(w, host0, budget_s=args.cpu_seconds)
+    print(json.dumps(line, default=float))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="wan1.3b_layer")
+    ap.add_argument("--sets", type=int, default=3, help="independent layer buffer sets used round-robin")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,229 @@
+/*
+ * pafu.h - C ABI of the PaFu-KV inference hot path on NVIDIA B200 (sm_100a).
+ *
+ * The path is the per-layer cache update and attention of the paper's inference
+ * procedure (Algorithm 2; Sec. 3.3, 3.4):
+ *
+ *     score   -> salience of every cached token from the S-MLP head
+ *     select  -> indices of the retained tokens (sink + top-k salient + recent)
+ *     compact -> KV <- Select(KV; ids), SL <- Select(SL; ids)
+ *     attend  -> the new chunk's queries over [retained cache ; chunk's own tokens]
+ *
+ * Conventions that hold for every entry point
+ *   - Plain C; every function returns a pafu_status and never throws or aborts.
+ *   - No function allocates or frees device memory and none synchronises the device,
+ *     unless its comment says otherwise.  All GPU work is enqueued on the caller's CUDA
+ *     stream, passed as `void*` (a cudaStream_t; NULL is the default stream).
+ *   - The caller owns every buffer.  "device" pointers are CUDA device pointers valid
+ *     on the current device; "host" pointers are ordinary host memory read before the
+ *     call returns.  Device buffers must be 16-byte aligned.
+ *   - bf16 tensors are raw 16-bit patterns (`uint16_t`).  Token tensors are token-major
+ *     `[tokens, n_heads, d_head]`, contiguous (d_model = n_heads * d_head elements per
+ *     row) - the merged layout the paper feeds to the S-MLP (Appendix A, "S-MLP").
+ *   - Several independent streams (a ragged batch) are packed back to back: stream s owns
+ *     token rows [cu[s], cu[s+1]) of a tensor, `cu` being a host prefix array of
+ *     n_streams + 1 entries starting at 0.  At most PAFU_MAX_STREAMS streams.
+ *   - Argument errors are found on the host before anything is launched; in that case no
+ *     output is touched.
+ *   - Kernels that wait on asynchronous copies bound every wait.  A wait that runs out
+ *     records a code in the workspace header and the kernel returns; see
+ *     pafu_workspace_status().
+ */
+#ifndef PAFU_H_
+#define PAFU_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PAFU_MAX_STREAMS 32
+
+typedef int32_t pafu_status;
+enum {
+    PAFU_OK = 0,
+    PAFU_ERR_INVALID_ARG = 1,        /* null pointer, negative size, bad enum, bad prefix array */
+    PAFU_ERR_BAD_BUDGET = 2,         /* negative budget / sink / recent */
+    PAFU_ERR_UNSUPPORTED_SHAPE = 3,  /* a dimension outside the supported set (see each call) */
+    PAFU_ERR_WORKSPACE_TOO_SMALL = 4,
+    PAFU_ERR_MISALIGNED = 5,         /* a device pointer is not 16-byte aligned */
+    PAFU_ERR_CUDA = 6,               /* a CUDA runtime/driver call failed (launch error, no device) */
+    PAFU_ERR_TIMEOUT = 7             /* a bounded device-side wait ran out (pafu_workspace_status) */
+};
+
+/* Activation between the two linear layers of the salience head. */
+enum { PAFU_ACT_GELU = 0 /* x * Phi(x), exact erf form */, PAFU_ACT_SILU = 1 /* paper's S-MLP */ };
+/* Map applied to the mean of the head's outputs. */
+enum { PAFU_FINAL_NONE = 0, PAFU_FINAL_SIGMOID = 1 };
+
+/* Geometry of one call.  cu_T: cache tokens per stream before pruning; cu_Lq: chunk (query)
+ * tokens per stream.  Both are HOST arrays of n_streams + 1 non-decreasing prefix offsets.
+ * A function that does not need one of them ignores it (may be NULL). */
+typedef struct pafu_shape {
+    int32_t n_heads;
+    int32_t d_head;
+    int32_t n_streams;
+    const int64_t* cu_T;   /* host */
+    const int64_t* cu_Lq;  /* host */
+} pafu_shape;
+
+/* Salience Estimation Head (Sec. 3.3; Appendix A "S-MLP"): two linear layers with an
+ * activation in between; the d_out outputs are averaged into one scalar per token.
+ * Weights use the torch.nn.Linear layout.  All four pointers are DEVICE bf16 arrays;
+ * b1 and b2 may be NULL (no bias).  The paper's head is d_in = 4608, d_hidden = 1024,
+ * d_out = 12, SiLU, no final map. */
+typedef struct pafu_head {
+    int32_t d_in;
+    int32_t d_hidden;
+    int32_t d_out;
+    int32_t act;           /* PAFU_ACT_* */
+    int32_t final;         /* PAFU_FINAL_* */
+    const uint16_t* w1;    /* device [d_hidden, d_in] */
+    const uint16_t* b1;    /* device [d_hidden] or NULL */
+    const uint16_t* w2;    /* device [d_out, d_hidden] */
+    const uint16_t* b2;    /* device [d_out] or NULL */
+} pafu_head;
+
+/* Retention rule of one stream, in absolute token counts. */
+typedef struct pafu_policy {
+    int64_t n_sink;    /* leading tokens always kept (frame sink, Sec. 4.1) */
+    int64_t n_recent;  /* trailing tokens always kept (the newest chunk survives one round, Alg. 2) */
+    int64_t budget;    /* tokens kept in total; T <= budget keeps all T */
+} pafu_policy;
+
+/* Library version (major * 1000 + minor). */
+int32_t pafu_version(void);
+
+/* Static, human-readable name of a status code. */
+const char* pafu_status_string(pafu_status s);
+
+/* Number of tokens each stream keeps, as a prefix array.
+ * cu_B (HOST, out, n_streams + 1 entries): cu_B[0] = 0, cu_B[s+1] - cu_B[s] = min(budget_s, T_s).
+ * `policy` is a HOST array of n_streams entries.  Pure host arithmetic. */
+pafu_status pafu_kept_counts(const pafu_shape* shape, const pafu_policy* policy, int64_t* cu_B);
+
+/* Bytes of device scratch that pafu_score / pafu_select / pafu_chunk_attn / pafu_step need
+ * for this geometry (`head` and `policy` may be NULL when the corresponding step is not
+ * used).  Returns 0 on invalid arguments.  The workspace must be 256-byte aligned; its
+ * first 256 bytes are a status header which the caller zeroes once after allocating. */
+size_t pafu_workspace_bytes(const pafu_shape* shape, const pafu_policy* policy,
+                            const pafu_head* head);
+
+/* Reads the workspace's status header.  SYNCHRONISES `stream` (one 4-byte device-to-host
+ * copy).  Returns PAFU_OK, or PAFU_ERR_TIMEOUT if a kernel gave up on a bounded wait since
+ * the header was last zeroed (the outputs of that launch are then undefined). */
+pafu_status pafu_workspace_status(const void* ws, void* stream);
+
+/* Step 1 - salience scores (Sec. 3.3, 3.4; Appendix A "S-MLP").
+ * For every token row x of X: h = act(W1 x + b1); y = W2 h + b2; s = mean_o y_o;
+ * s <- sigmoid(s) if head->final == PAFU_FINAL_SIGMOID.  bf16 operands, fp32 accumulation,
+ * fp32 activation and output.
+ *   head      HOST struct with DEVICE weight pointers
+ *   X         device bf16 [n_tokens, ldx], row stride ldx >= d_in elements, ldx % 8 == 0
+ *   scores    device fp32 [n_tokens], out
+ *   ws        device workspace (pafu_workspace_bytes), ws_bytes its size
+ * Supported: d_in % 64 == 0, d_hidden % 16 == 0 and <= 1024, d_out >= 1.
+ * n_tokens == 0 is a no-op. */
+pafu_status pafu_score(const pafu_head* head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
+                       float* scores, void* ws, size_t ws_bytes, void* stream);
+
+/* Step 2 - retained indices (Sec. 3.4 inference paragraph; Algorithm 2 "Top-k"; frame sink
+ * Sec. 4.1).  Per stream with T tokens and (n_sink, n_recent, budget):
+ *   T <= budget            : keep all T tokens;
+ *   else n_recent' = min(n_recent, budget), n_sink' = min(n_sink, budget - n_recent'),
+ *        k = budget - n_sink' - n_recent', and the kept set is
+ *        [0, n_sink') U top-k of scores[n_sink' : T - n_recent') U [T - n_recent', T).
+ * Ranking is by fp32 value, higher first; equal values (-0 == +0) go to the lower index;
+ * NaN ranks below every number.  The result is exact and deterministic.
+ *   scores    device fp32 [cu_T[n_streams]], packed over streams
+ *   policy    HOST array [n_streams]
+ *   idx       device int32 [cu_B[n_streams]], out: per stream, stream-local token indices
+ *             in strictly ascending order at offset cu_B[s] (cu_B from pafu_kept_counts)
+ * Each stream needs T < 2^31. */
+pafu_status pafu_select(const float* scores, const pafu_shape* shape, const pafu_policy* policy,
+                        int32_t* idx, void* ws, size_t ws_bytes, void* stream);
+
+/* Step 3 - KV <- Select(KV; ids), SL <- Select(SL; ids) (Algorithm 2).
+ * For stream s and i in [0, B_s): Kc[cu_B[s] + i, :] = K[cu_T[s] + idx[cu_B[s] + i], :], same
+ * for V and, when SL and SLc are both non-NULL, for the fp32 salience list.  Raw copies,
+ * bit exact.  Out of place: outputs must not overlap inputs.
+ *   K, V      device bf16 [cu_T[n_streams], n_heads, d_head]
+ *   idx       device int32 as written by pafu_select (values must lie in [0, T_s))
+ *   Kc, Vc    device bf16 [cu_B[n_streams], n_heads, d_head], out
+ * Supported: n_heads * d_head % 8 == 0. */
+pafu_status pafu_compact(const uint16_t* K, const uint16_t* V, const float* SL, const int32_t* idx,
+                         const pafu_shape* shape, const pafu_policy* policy,
+                         uint16_t* Kc, uint16_t* Vc, float* SLc, void* stream);
+
+/* Step 4 - chunk attention over the retained cache (Sec. 3.2 for the operator
+ * P = softmax(Q K^T / sqrt(D)); Eq. 2 / Eq. 7 for what it ranges over).
+ * Per stream s, head n, query row i: o_i = sum_j softmax_j(scale * q_i . k_j) v_j where j runs
+ * over the B_s retained tokens (Kc, Vc) and then the stream's own Lq_s chunk tokens (Kq, Vq).
+ * No mask: the chunk is bidirectional and sees the whole retained cache.  bf16 operands,
+ * fp32 accumulation and softmax; probabilities are rounded to bf16 before the P V product.
+ *   Q         device bf16 [cu_Lq[n_streams], n_heads, d_head]
+ *   Kc, Vc    device bf16 [cu_B[n_streams], n_heads, d_head]
+ *   cu_B      HOST prefix array [n_streams + 1] of retained tokens
+ *   Kq, Vq    device bf16 [cu_Lq[n_streams], n_heads, d_head]; both NULL = no chunk segment
+ *   scale     softmax scale; 0 means 1 / sqrt(d_head)
+ *   O         device bf16 [cu_Lq[n_streams], n_heads, d_head], out
+ *   LSE       device fp32 [n_heads, cu_Lq[n_streams]] log-sum-exp of the scaled logits, or NULL
+ * A query with no keys at all gets o = 0 and LSE = -inf.  Supported: d_head in {64, 128}. */
+pafu_status pafu_chunk_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
+                            const int64_t* cu_B, const uint16_t* Kq, const uint16_t* Vq,
+                            const pafu_shape* shape, float scale, uint16_t* O, float* LSE,
+                            void* ws, size_t ws_bytes, void* stream);
+
+/* Arguments of one whole layer step (Algorithm 2's order: score, Top-k, Select, attend). */
+typedef struct pafu_step_args {
+    pafu_shape shape;
+    const pafu_head* head;        /* host struct, device weights; d_in must equal n_heads*d_head */
+    const pafu_policy* policy;    /* host [n_streams] */
+    const uint16_t* K;            /* device [cu_T[n], N, D]: cache keys, also the head's input */
+    const uint16_t* V;            /* device [cu_T[n], N, D] */
+    const uint16_t* Q;            /* device [cu_Lq[n], N, D] */
+    const uint16_t* Kq;           /* device [cu_Lq[n], N, D] */
+    const uint16_t* Vq;           /* device [cu_Lq[n], N, D] */
+    float scale;                  /* 0 = 1/sqrt(D) */
+    float* scores;                /* device fp32 [cu_T[n]], out (also the salience list SL) */
+    int32_t* idx;                 /* device int32 [cu_B[n]], out */
+    uint16_t* Kc;                 /* device [cu_B[n], N, D], out */
+    uint16_t* Vc;                 /* device [cu_B[n], N, D], out */
+    float* SLc;                   /* device fp32 [cu_B[n]], out, or NULL */
+    uint16_t* O;                  /* device [cu_Lq[n], N, D], out */
+    float* LSE;                   /* device fp32 [N, cu_Lq[n]], out, or NULL */
+    void* ws;                     /* device workspace */
+    size_t ws_bytes;
+} pafu_step_args;
+
+/* Step 5 - the four steps in order on one stream.  Produces exactly what pafu_score,
+ * pafu_select, pafu_compact and pafu_chunk_attn produce when called in sequence with the
+ * same buffers (the salience head reads each token's K across all heads). */
+pafu_status pafu_step(const pafu_step_args* args, void* stream);
+
+/* pafu_step with timestamps: identical launches, plus five caller-created CUDA events
+ * (HOST array of 5 cudaEvent_t passed as void*) recorded on `stream` before the score step and
+ * after the score, select, compact and attention steps.  Lets a caller attribute the step's
+ * time to its kernels without changing what runs. */
+pafu_status pafu_step_timed(const pafu_step_args* args, void* const* events, void* stream);
+
+/* Bytes of device memory pafu_step_host needs as its arena for this geometry. */
+size_t pafu_step_host_arena_bytes(const pafu_shape* shape, const pafu_policy* policy,
+                                  const pafu_head* head);
+
+/* pafu_step for callers whose tensors live in HOST memory.  Every tensor pointer in `args`
+ * (K, V, Q, Kq, Vq, the head's weights; outputs scores, idx, O and, if non-NULL, Kc, Vc, SLc,
+ * LSE) is a HOST pointer - pinned memory makes the copies asynchronous.  args->ws/ws_bytes
+ * are ignored.  The call copies the inputs into `arena` (device, 256-byte aligned, at least
+ * pafu_step_host_arena_bytes), runs pafu_step there, copies the outputs back and
+ * SYNCHRONISES `stream` before returning, so the host outputs are valid on return.
+ * Returns PAFU_ERR_TIMEOUT if a bounded device wait ran out. */
+pafu_status pafu_step_host(const pafu_step_args* args, void* arena, size_t arena_bytes,
+                           void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* PAFU_H_ */

@@ -1,0 +1,261 @@
+"""Thin ctypes binding of ``libpafu.so``: argument marshalling only.
+
+Functions carry the C names (``pafu_score`` ...).  Device tensors are torch CUDA tensors
+(bf16 for token tensors and weights, fp32 scores, int32 indices); the binding passes their
+``data_ptr()`` and the current CUDA stream.  There is no CPU path: loading fails loudly when
+the library has not been built, and every call raises ``PafuError`` on a non-zero status.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libpafu.so")
+
+PAFU_MAX_STREAMS = 32
+ACT_GELU, ACT_SILU = 0, 1
+FINAL_NONE, FINAL_SIGMOID = 0, 1
+
+STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET",
+                3: "PAFU_ERR_UNSUPPORTED_SHAPE", 4: "PAFU_ERR_WORKSPACE_TOO_SMALL",
+                5: "PAFU_ERR_MISALIGNED", 6: "PAFU_ERR_CUDA", 7: "PAFU_ERR_TIMEOUT"}
+
+EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
+           "pafu_workspace_status", "pafu_score", "pafu_select", "pafu_compact",
+           "pafu_chunk_attn", "pafu_step", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host"]
+
+
+class PafuError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = STATUS_NAMES.get(status, str(status))
+        try:
+            msg += " (%s)" % lib().pafu_status_string(status).decode()
+        except Exception:
+            pass
+        super().__init__("%s failed: %s" % (where, msg))
+
+
+class CShape(ctypes.Structure):
+    _fields_ = [("n_heads", ctypes.c_int32), ("d_head", ctypes.c_int32),
+                ("n_streams", ctypes.c_int32), ("cu_T", ctypes.c_void_p),
+                ("cu_Lq", ctypes.c_void_p)]
+
+
+class CHead(ctypes.Structure):
+    _fields_ = [("d_in", ctypes.c_int32), ("d_hidden", ctypes.c_int32), ("d_out", ctypes.c_int32),
+                ("act", ctypes.c_int32), ("final", ctypes.c_int32),
+                ("w1", ctypes.c_void_p), ("b1", ctypes.c_void_p),
+                ("w2", ctypes.c_void_p), ("b2", ctypes.c_void_p)]
+
+
+class CPolicy(ctypes.Structure):
+    _fields_ = [("n_sink", ctypes.c_int64), ("n_recent", ctypes.c_int64),
+                ("budget", ctypes.c_int64)]
+
+
+class CStepArgs(ctypes.Structure):
+    _fields_ = [("shape", CShape), ("head", ctypes.POINTER(CHead)),
+                ("policy", ctypes.POINTER(CPolicy)),
+                ("K", ctypes.c_void_p), ("V", ctypes.c_void_p), ("Q", ctypes.c_void_p),
+                ("Kq", ctypes.c_void_p), ("Vq", ctypes.c_void_p), ("scale", ctypes.c_float),
+                ("scores", ctypes.c_void_p), ("idx", ctypes.c_void_p), ("Kc", ctypes.c_void_p),
+                ("Vc", ctypes.c_void_p), ("SLc", ctypes.c_void_p), ("O", ctypes.c_void_p),
+                ("LSE", ctypes.c_void_p), ("ws", ctypes.c_void_p), ("ws_bytes", ctypes.c_size_t)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libpafu.so is missing at %s - build it with "
+                "`python -m paper_2601_21896_b200.build` (needs nvcc); there is no CPU path" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, i32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_size_t
+        L.pafu_version.restype = i32
+        L.pafu_version.argtypes = []
+        L.pafu_status_string.restype = ctypes.c_char_p
+        L.pafu_status_string.argtypes = [i32]
+        L.pafu_kept_counts.restype = i32
+        L.pafu_kept_counts.argtypes = [ctypes.POINTER(CShape), ctypes.POINTER(CPolicy), vp]
+        L.pafu_workspace_bytes.restype = sz
+        L.pafu_workspace_bytes.argtypes = [ctypes.POINTER(CShape), ctypes.POINTER(CPolicy),
+                                           ctypes.POINTER(CHead)]
+        L.pafu_workspace_status.restype = i32
+        L.pafu_workspace_status.argtypes = [vp, vp]
+        L.pafu_score.restype = i32
+        L.pafu_score.argtypes = [ctypes.POINTER(CHead), vp, i64, i64, vp, vp, sz, vp]
+        L.pafu_select.restype = i32
+        L.pafu_select.argtypes = [vp, ctypes.POINTER(CShape), ctypes.POINTER(CPolicy), vp, vp, sz, vp]
+        L.pafu_compact.restype = i32
+        L.pafu_compact.argtypes = [vp, vp, vp, vp, ctypes.POINTER(CShape), ctypes.POINTER(CPolicy),
+                                   vp, vp, vp, vp]
+        L.pafu_chunk_attn.restype = i32
+        L.pafu_chunk_attn.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.POINTER(CShape),
+                                      ctypes.c_float, vp, vp, vp, sz, vp]
+        L.pafu_step.restype = i32
+        L.pafu_step.argtypes = [ctypes.POINTER(CStepArgs), vp]
+        L.pafu_step_timed.restype = i32
+        L.pafu_step_timed.argtypes = [ctypes.POINTER(CStepArgs), ctypes.POINTER(vp), vp]
+        L.pafu_step_host_arena_bytes.restype = sz
+        L.pafu_step_host_arena_bytes.argtypes = [ctypes.POINTER(CShape), ctypes.POINTER(CPolicy),
+                                                 ctypes.POINTER(CHead)]
+        L.pafu_step_host.restype = i32
+        L.pafu_step_host.argtypes = [ctypes.POINTER(CStepArgs), vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+# ------------------------------------------------------------------------- marshalling
+def _ptr(t) -> Optional[int]:
+    """Address of a torch tensor (device or host) / numpy array, or None."""
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        assert t.is_contiguous(), "tensor must be contiguous"
+        return t.data_ptr()
+    if isinstance(t, np.ndarray):
+        assert t.flags["C_CONTIGUOUS"]
+        return t.ctypes.data
+    raise TypeError(type(t))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise PafuError(status, where)
+
+
+class Shape:
+    """Host-side geometry: keeps the prefix arrays alive for the duration of a call."""
+
+    def __init__(self, n_heads: int, d_head: int, cu_T: Optional[Sequence[int]] = None,
+                 cu_Lq: Optional[Sequence[int]] = None, n_streams: Optional[int] = None):
+        self.cu_T = None if cu_T is None else np.ascontiguousarray(cu_T, dtype=np.int64)
+        self.cu_Lq = None if cu_Lq is None else np.ascontiguousarray(cu_Lq, dtype=np.int64)
+        if n_streams is None:
+            ref = self.cu_T if self.cu_T is not None else self.cu_Lq
+            n_streams = len(ref) - 1
+        self.n_heads, self.d_head, self.n_streams = n_heads, d_head, n_streams
+        self.c = CShape(n_heads, d_head, n_streams, _ptr(self.cu_T), _ptr(self.cu_Lq))
+
+
+class Head:
+    """Salience head: device bf16 weights in torch.nn.Linear layout."""
+
+    def __init__(self, w1, b1, w2, b2, act: int = ACT_GELU, final: int = FINAL_NONE,
+                 dims: Optional[Sequence[int]] = None):
+        self.tensors = (w1, b1, w2, b2)
+        if dims is None:
+            dims = (w1.shape[1], w1.shape[0], w2.shape[0])
+        self.c = CHead(int(dims[0]), int(dims[1]), int(dims[2]), act, final,
+                       _ptr(w1), _ptr(b1), _ptr(w2), _ptr(b2))
+
+
+def make_policy(n_sink, n_recent, budget, n_streams: int):
+    """ctypes array of per-stream policies; scalars are broadcast."""
+    def seq(v):
+        return list(v) if isinstance(v, (list, tuple, np.ndarray)) else [v] * n_streams
+    arr = (CPolicy * n_streams)()
+    for s, (a, b, c) in enumerate(zip(seq(n_sink), seq(n_recent), seq(budget))):
+        arr[s] = CPolicy(int(a), int(b), int(c))
+    return arr
+
+
+# ------------------------------------------------------------------------------ entry points
+def pafu_version() -> int:
+    return lib().pafu_version()
+
+
+def pafu_kept_counts(shape: Shape, policy) -> np.ndarray:
+    cu_B = np.zeros(shape.n_streams + 1, dtype=np.int64)
+    _check(lib().pafu_kept_counts(ctypes.byref(shape.c), policy, _ptr(cu_B)), "pafu_kept_counts")
+    return cu_B
+
+
+def pafu_workspace_bytes(shape: Shape, policy=None, head: Optional[Head] = None) -> int:
+    return lib().pafu_workspace_bytes(ctypes.byref(shape.c), policy,
+                                      ctypes.byref(head.c) if head is not None else None)
+
+
+def pafu_workspace_status(ws: torch.Tensor) -> int:
+    return lib().pafu_workspace_status(_ptr(ws), _stream())
+
+
+def pafu_score(head: Head, X: torch.Tensor, scores: torch.Tensor, ws: Optional[torch.Tensor] = None,
+               n_tokens: Optional[int] = None, ldx: Optional[int] = None) -> None:
+    n = X.shape[0] if n_tokens is None else n_tokens
+    ld = (X.numel() // max(X.shape[0], 1)) if ldx is None else ldx
+    _check(lib().pafu_score(ctypes.byref(head.c), _ptr(X), n, ld, _ptr(scores), _ptr(ws),
+                            0 if ws is None else ws.numel() * ws.element_size(), _stream()),
+           "pafu_score")
+
+
+def pafu_select(scores: torch.Tensor, shape: Shape, policy, idx: torch.Tensor,
+                ws: Optional[torch.Tensor] = None) -> None:
+    _check(lib().pafu_select(_ptr(scores), ctypes.byref(shape.c), policy, _ptr(idx), _ptr(ws),
+                             0 if ws is None else ws.numel() * ws.element_size(), _stream()),
+           "pafu_select")
+
+
+def pafu_compact(K, V, SL, idx, shape: Shape, policy, Kc, Vc, SLc) -> None:
+    _check(lib().pafu_compact(_ptr(K), _ptr(V), _ptr(SL), _ptr(idx), ctypes.byref(shape.c), policy,
+                              _ptr(Kc), _ptr(Vc), _ptr(SLc), _stream()), "pafu_compact")
+
+
+def pafu_chunk_attn(Q, Kc, Vc, cu_B, Kq, Vq, shape: Shape, scale: float, O, LSE=None,
+                    ws: Optional[torch.Tensor] = None) -> None:
+    cu_B = np.ascontiguousarray(cu_B, dtype=np.int64)
+    _check(lib().pafu_chunk_attn(_ptr(Q), _ptr(Kc), _ptr(Vc), _ptr(cu_B), _ptr(Kq), _ptr(Vq),
+                                 ctypes.byref(shape.c), float(scale), _ptr(O), _ptr(LSE), _ptr(ws),
+                                 0 if ws is None else ws.numel() * ws.element_size(), _stream()),
+           "pafu_chunk_attn")
+
+
+def step_args(shape: Shape, head: Head, policy, K, V, Q, Kq, Vq, scale, scores, idx, Kc, Vc, SLc,
+              O, LSE, ws) -> CStepArgs:
+    args = CStepArgs(shape.c, ctypes.pointer(head.c), ctypes.cast(policy, ctypes.POINTER(CPolicy)),
+                     _ptr(K), _ptr(V), _ptr(Q), _ptr(Kq), _ptr(Vq), float(scale), _ptr(scores),
+                     _ptr(idx), _ptr(Kc), _ptr(Vc), _ptr(SLc), _ptr(O), _ptr(LSE), _ptr(ws),
+                     0 if ws is None else ws.numel() * ws.element_size())
+    args._keep = (shape, head, policy)   # the struct only holds raw pointers into these
+    return args
+
+
+def pafu_step(args: CStepArgs) -> None:
+    _check(lib().pafu_step(ctypes.byref(args), _stream()), "pafu_step")
+
+
+def event_handles(events: Sequence["torch.cuda.Event"]):
+    """ctypes array of the cudaEvent_t handles of five torch timing events (each must have
+    been recorded once so that torch has created it)."""
+    arr = (ctypes.c_void_p * 5)()
+    for i, e in enumerate(events):
+        arr[i] = e.cuda_event
+    return arr
+
+
+def pafu_step_timed(args: CStepArgs, handles) -> None:
+    _check(lib().pafu_step_timed(ctypes.byref(args), handles, _stream()), "pafu_step_timed")
+
+
+def pafu_step_host_arena_bytes(shape: Shape, policy, head: Head) -> int:
+    return lib().pafu_step_host_arena_bytes(ctypes.byref(shape.c), policy, ctypes.byref(head.c))
+
+
+def pafu_step_host(args: CStepArgs, arena: torch.Tensor) -> None:
+    _check(lib().pafu_step_host(ctypes.byref(args), _ptr(arena),
+                                arena.numel() * arena.element_size(), _stream()), "pafu_step_host")

@@ -1,0 +1,44 @@
+// Internal declarations shared by the kernels' launchers and the C ABI layer.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/pafu.h"
+
+namespace pafu {
+
+// Per-stream prefix offsets and retention parameters, passed to kernels by value.
+struct StreamTable {
+    int32_t n_streams;
+    int64_t cu_T[PAFU_MAX_STREAMS + 1];   // cache tokens
+    int64_t cu_B[PAFU_MAX_STREAMS + 1];   // retained tokens
+    int64_t cu_Lq[PAFU_MAX_STREAMS + 1];  // chunk tokens
+    int64_t n_sink[PAFU_MAX_STREAMS];     // clamped sink length
+    int64_t n_recent[PAFU_MAX_STREAMS];   // clamped recent length
+    int64_t k[PAFU_MAX_STREAMS];          // candidates to take by salience
+};
+
+// Workspace layout: [0, 256) status header (int32 words), then per-step scratch.
+constexpr size_t kWsHeaderBytes = 256;
+constexpr int kStatusWordTimeout = 0;   // non-zero: a bounded wait ran out
+
+inline pafu_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? PAFU_OK : PAFU_ERR_CUDA; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Launchers (each enqueues on `stream` and returns the launch status).
+pafu_status launch_score(const pafu_head& head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
+                         float* scores, void* ws, size_t ws_bytes, cudaStream_t stream);
+pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* idx,
+                          cudaStream_t stream);
+pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL,
+                           const int32_t* idx, const StreamTable& st, int32_t d_model,
+                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream);
+pafu_status launch_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
+                        const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
+                        int32_t n_heads, int32_t d_head, float scale, uint16_t* O, float* LSE,
+                        void* ws, size_t ws_bytes, cudaStream_t stream);
+size_t attn_workspace_bytes(const StreamTable& st, int32_t n_heads, int32_t d_head);
+size_t score_workspace_bytes(const pafu_head& head);
+
+}  // namespace pafu

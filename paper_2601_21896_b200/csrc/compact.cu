@@ -1,0 +1,70 @@
+// KV <- Select(KV; ids), SL <- Select(SL; ids) (Algorithm 2): row gather of the kept tokens.
+//
+// HBM-bound copy.  One warp moves one kept token: its K row and its V row (d_model bf16 each)
+// in 16-byte pieces, all loads of a batch issued before the first store so that each warp
+// keeps up to 12 x 512 B in flight.  Rows are contiguous, so every access is fully coalesced;
+// the only indirection is one int32 index per row.
+#include "common.cuh"
+
+namespace pafu {
+
+constexpr int kCompactWarpsPerBlock = 8;
+constexpr int kCompactUnroll = 6;   // 6 x 32 lanes x 16 B = one 3072-byte row (d_model 1536)
+
+__device__ __forceinline__ uint4 ld_nc_v4(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__global__ void __launch_bounds__(kCompactWarpsPerBlock * 32)
+compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
+                    const float* __restrict__ SL, const int32_t* __restrict__ idx,
+                    StreamTable st, int32_t chunks_per_row,
+                    uint4* __restrict__ Kc, uint4* __restrict__ Vc, float* __restrict__ SLc,
+                    int64_t n_rows) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = (int64_t)blockIdx.x * kCompactWarpsPerBlock + (threadIdx.x >> 5);
+    const int64_t n_warps = (int64_t)gridDim.x * kCompactWarpsPerBlock;
+    for (int64_t r = warp0; r < n_rows; r += n_warps) {
+        int s = 0;
+        while (s + 1 < st.n_streams && r >= st.cu_B[s + 1]) ++s;
+        const int64_t src_row = st.cu_T[s] + (int64_t)__ldg(idx + r);
+        const uint4* ks = K + src_row * chunks_per_row;
+        const uint4* vs = V + src_row * chunks_per_row;
+        uint4* kd = Kc + r * chunks_per_row;
+        uint4* vd = Vc + r * chunks_per_row;
+        for (int c0 = 0; c0 < chunks_per_row; c0 += 32 * kCompactUnroll) {
+            uint4 kb[kCompactUnroll], vb[kCompactUnroll];
+#pragma unroll
+            for (int u = 0; u < kCompactUnroll; ++u) {
+                const int c = c0 + u * 32 + lane;
+                if (c < chunks_per_row) { kb[u] = ld_nc_v4(ks + c); vb[u] = ld_nc_v4(vs + c); }
+            }
+#pragma unroll
+            for (int u = 0; u < kCompactUnroll; ++u) {
+                const int c = c0 + u * 32 + lane;
+                if (c < chunks_per_row) { kd[c] = kb[u]; vd[c] = vb[u]; }
+            }
+        }
+        if (SLc != nullptr && lane == 0) SLc[r] = __ldg(SL + src_row);
+    }
+}
+
+pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL,
+                           const int32_t* idx, const StreamTable& st, int32_t d_model,
+                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream) {
+    const int64_t n_rows = st.cu_B[st.n_streams];
+    if (n_rows == 0) return PAFU_OK;
+    const int32_t chunks = d_model / 8;
+    int64_t blocks = (n_rows + kCompactWarpsPerBlock - 1) / kCompactWarpsPerBlock;
+    const int64_t max_blocks = 148 * 8 * 4;   // a few resident waves; larger inputs loop
+    if (blocks > max_blocks) blocks = max_blocks;
+    compact_rows_kernel<<<(unsigned)blocks, kCompactWarpsPerBlock * 32, 0, stream>>>(
+        reinterpret_cast<const uint4*>(K), reinterpret_cast<const uint4*>(V), SL, idx, st, chunks,
+        reinterpret_cast<uint4*>(Kc), reinterpret_cast<uint4*>(Vc), SLc, n_rows);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace pafu

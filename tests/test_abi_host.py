@@ -1,0 +1,101 @@
+"""Host-side checks that need no GPU: the C-ABI library loads, exports every symbol the
+header declares, and rejects bad arguments on the host before anything is launched."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2601_21896_b200 as pafu
+from paper_2601_21896_b200 import binding as B
+from paper_2601_21896_b200 import build as pbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    pbuild.build_library()
+    return B.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "pafu.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(pafu_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(L):
+    names = declared_functions()
+    assert set(names) == set(B.EXPORTS), (names, B.EXPORTS)
+    for n in names:
+        assert getattr(L, n) is not None
+    assert L.pafu_version() >= 1000
+    assert L.pafu_status_string(0) == b"ok"
+    assert L.pafu_status_string(7) == b"bounded device wait ran out"
+
+
+def test_struct_layouts_match_header():
+    # the ctypes mirrors must have the C layout (LP64): sizes pin padding mistakes
+    assert ctypes.sizeof(B.CShape) == 32
+    assert ctypes.sizeof(B.CHead) == 56
+    assert ctypes.sizeof(B.CPolicy) == 24
+    assert ctypes.sizeof(B.CStepArgs) == 32 + 8 + 8 + 5 * 8 + 8 + 7 * 8 + 8 + 8
+
+
+def test_kept_counts_and_clamping(L):
+    sh = pafu.Shape(12, 128, [0, 28080, 28080 + 100, 28080 + 100 + 50], None)
+    pol = pafu.make_policy(1560, 4680, [14040, 200, 7], 3)
+    assert pafu.pafu_kept_counts(sh, pol).tolist() == [0, 14040, 14140, 14147]
+    with pytest.raises(pafu.PafuError) as e:
+        pafu.pafu_kept_counts(sh, pafu.make_policy(1, 1, [5, -1, 5], 3))
+    assert e.value.status == 2
+    with pytest.raises(pafu.PafuError) as e:
+        pafu.pafu_kept_counts(pafu.Shape(1, 64, [0, 5, 3], None), pafu.make_policy(0, 0, 1, 2))
+    assert e.value.status == 1   # prefix array not monotone
+
+
+def test_argument_errors_are_caught_on_the_host(L):
+    vp = ctypes.c_void_p
+    sh = pafu.Shape(2, 64, [0, 512], [0, 64])
+    pol = pafu.make_policy(4, 64, 128, 1)
+    fake = 0x10000   # never dereferenced: every call below must fail before launching
+    head = B.CHead(128, 32, 1, 0, 0, fake, None, fake, None)
+    assert L.pafu_score(None, fake, 4, 128, fake, None, 0, None) == 1
+    assert L.pafu_score(ctypes.byref(head), None, 4, 128, fake, None, 0, None) == 1
+    assert L.pafu_score(ctypes.byref(head), fake, -1, 128, fake, None, 0, None) == 1
+    assert L.pafu_score(ctypes.byref(head), fake, 4, 64, fake, None, 0, None) == 1       # ldx < d_in
+    assert L.pafu_score(ctypes.byref(head), fake + 2, 4, 128, fake, None, 0, None) == 5   # misaligned
+    assert L.pafu_score(ctypes.byref(head), fake, 0, 128, fake, None, 0, None) == 0       # empty: no-op
+    bad = B.CHead(100, 32, 1, 0, 0, fake, None, fake, None)
+    assert L.pafu_score(ctypes.byref(bad), fake, 4, 128, fake, None, 0, None) == 3
+    bad = B.CHead(128, 32, 1, 7, 0, fake, None, fake, None)
+    assert L.pafu_score(ctypes.byref(bad), fake, 4, 128, fake, None, 0, None) == 1
+    assert L.pafu_select(None, ctypes.byref(sh.c), pol, fake, None, 0, None) == 1
+    assert L.pafu_select(fake, ctypes.byref(sh.c), None, fake, None, 0, None) == 1
+    assert L.pafu_select(fake, ctypes.byref(sh.c), pafu.make_policy(-1, 0, 5, 1), fake, None, 0, None) == 2
+    assert L.pafu_select(fake, None, pol, fake, None, 0, None) == 1
+    assert L.pafu_compact(fake, fake, None, fake, ctypes.byref(sh.c), pol, fake, fake + 4096, None, None) == 1  # aliasing
+    assert L.pafu_compact(fake, fake + 4096, None, None, ctypes.byref(sh.c), pol, fake + 8192, fake + 12288, None, None) == 1
+    assert L.pafu_compact(fake, fake + 4096, fake, fake, ctypes.byref(sh.c), pol, fake + 8192, fake + 12288, None, None) == 1
+    cu_B = np.array([0, 128], dtype=np.int64)
+    sh3 = pafu.Shape(2, 96, [0, 512], [0, 64])
+    assert L.pafu_chunk_attn(fake, fake, fake, cu_B.ctypes.data, fake, fake, ctypes.byref(sh3.c), 0.0, fake, None, None, 0, None) == 3
+    assert L.pafu_chunk_attn(fake, fake, fake, cu_B.ctypes.data, fake, None, ctypes.byref(sh.c), 0.0, fake, None, None, 0, None) == 1
+    assert L.pafu_chunk_attn(fake, fake, fake, cu_B.ctypes.data, fake, fake, ctypes.byref(sh.c), -1.0, fake, None, None, 0, None) == 1
+    assert L.pafu_chunk_attn(fake, fake, fake, None, fake, fake, ctypes.byref(sh.c), 0.0, fake, None, None, 0, None) == 1
+    too_many = pafu.Shape(2, 64, list(range(0, 35)), list(range(0, 35)))
+    assert L.pafu_select(fake, ctypes.byref(too_many.c), pafu.make_policy(0, 0, 1, 34), fake, None, 0, None) == 3
+    assert L.pafu_step(None, None) == 1
+    assert L.pafu_workspace_status(None, None) == 1
+    assert L.pafu_workspace_bytes(None, None, None) == 0
+    assert L.pafu_workspace_bytes(ctypes.byref(sh.c), pol, None) >= 256
+    assert L.pafu_workspace_bytes(ctypes.byref(sh.c), pol, None) % 256 == 0
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU path"):
+        B.lib()

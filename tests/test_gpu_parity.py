@@ -1,0 +1,275 @@
+"""GPU parity: every step of the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.  Integer and byte results must be bit exact; scores and attention
+outputs must agree within max-abs 2e-2 and mean-abs 2e-3 (bf16 inputs, fp32 accumulation)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2601_21896_b200 as pafu
+from paper_2601_21896_b200 import workloads as wl
+from paper_2601_21896_b200.harness import Layer, bf16_to_bits, to_device_bf16
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+
+
+def close(got, want, what=""):
+    got = np.asarray(got, dtype=np.float64); want = np.asarray(want, dtype=np.float64)
+    assert got.shape == want.shape, (got.shape, want.shape)
+    if got.size == 0:
+        return
+    assert np.all(np.isfinite(got)), what
+    err = np.abs(got - want)
+    assert err.max() <= MAX_ABS, (what, err.max(), np.unravel_index(err.argmax(), err.shape))
+    assert err.mean() <= MEAN_ABS, (what, err.mean())
+
+
+def oracle_scores(w, d):
+    return oracle.score(d["K"].reshape(d["K"].shape[0], -1), d["w1"], d["b1"], d["w2"], d["b2"],
+                        w.act, w.final)
+
+
+def oracle_select_streams(scores, w):
+    cuT = w.cu("T")
+    return [oracle.select(scores[cuT[s]:cuT[s + 1]], w.n_sink, w.n_recent, w.budget[s])
+            for s in range(w.n_streams)]
+
+
+def oracle_attn_streams(w, d, Kc_bits, Vc_bits, cu_B, rows=None):
+    cuQ = w.cu("Lq")
+    outs = []
+    for s in range(w.n_streams):
+        q = d["Q"][cuQ[s]:cuQ[s + 1]]
+        r = None if rows is None else rows[s]
+        O, L = oracle.attention(q, Kc_bits[cu_B[s]:cu_B[s + 1]], Vc_bits[cu_B[s]:cu_B[s + 1]],
+                                d["Kq"][cuQ[s]:cuQ[s + 1]], d["Vq"][cuQ[s]:cuQ[s + 1]], rows=r)
+        outs.append((O, L))
+    return outs
+
+
+SMALL = [wl.tiny(), wl.small_ragged(2, 128), wl.small_ragged(3, 64)]
+
+
+# --------------------------------------------------------------------------------- score
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: "%s-d%d" % (w.name, w.d_head))
+def test_score_matches_oracle(w):
+    d = wl.make_layer(w)
+    L = Layer(w, d)
+    L.score()
+    L.check_status()
+    close(L.scores[: L.nT].cpu().numpy(), oracle_scores(w, d), "score")
+
+
+@pytest.mark.parametrize("act,final,d_out,d_hidden,n", [
+    (wl.ACT_SILU, wl.FINAL_NONE, 12, 1024, 300),     # the paper's S-MLP widths (Appendix A)
+    (wl.ACT_GELU, wl.FINAL_SIGMOID, 1, 32, 129),
+    (wl.ACT_GELU, wl.FINAL_NONE, 3, 272, 1),
+    (wl.ACT_SILU, wl.FINAL_SIGMOID, 1, 256, 517),
+])
+def test_score_head_variants(act, final, d_out, d_hidden, n):
+    rng = np.random.default_rng(5)
+    d_in = 384
+    bits = lambda shape, s=1.0: wl.f32_to_bf16_bits((rng.standard_normal(shape) * s).astype(np.float32))
+    X = bits((n, d_in)); w1 = bits((d_hidden, d_in), d_in ** -0.5); b1 = bits((d_hidden,), 0.3)
+    w2 = bits((d_out, d_hidden), d_hidden ** -0.5); b2 = bits((d_out,), 0.3)
+    for use_bias in (True, False):
+        dev = [to_device_bf16(a) for a in (X, w1, b1, w2, b2)]
+        head = pafu.Head(dev[1], dev[2] if use_bias else None, dev[3], dev[4] if use_bias else None,
+                         act, final)
+        shape = pafu.Shape(3, 128, [0, n], [0, 1])
+        ws = torch.zeros(pafu.pafu_workspace_bytes(shape, None, head), dtype=torch.uint8, device="cuda")
+        out = torch.full((n,), float("nan"), device="cuda")
+        pafu.pafu_score(head, dev[0], out, ws)
+        assert pafu.pafu_workspace_status(ws) == 0
+        want = oracle.score(X, w1, b1 if use_bias else None, w2, b2 if use_bias else None, act, final)
+        close(out.cpu().numpy(), want, "score variant")
+
+
+# -------------------------------------------------------------------------------- select
+@pytest.mark.parametrize("kind", ["normal", "ties", "equal", "saturated", "heavy", "signed_zero"])
+def test_select_bit_exact(kind):
+    cases = [((512,), 4, 64, (128,)), ((1000, 37, 2048, 5), 3, 10, (500, 20, 1024, 9)),
+             ((4097,), 0, 0, (1,)), ((4097,), 0, 0, (4096,)), ((3000,), 100, 200, (250,)),
+             ((3000,), 5000, 0, (1000,)), ((1, 2, 3), 1, 1, (0, 1, 2)), ((28080,), 1560, 4680, (14040,)),
+             ((93600,), 1560, 4680, (9360,))]
+    for ci, (T, ns, nr, Bs) in enumerate(cases):
+        n = len(T)
+        cuT = np.concatenate([[0], np.cumsum(T)])
+        s = wl.random_scores(int(cuT[-1]), seed=ci, kind=kind, tag=ci)
+        if kind == "heavy":
+            s[::97] = np.nan; s[5::101] = np.inf; s[7::103] = -np.inf
+        shape = pafu.Shape(1, 64, cuT, None)
+        pol = pafu.make_policy(ns, nr, list(Bs), n)
+        cu_B = pafu.pafu_kept_counts(shape, pol)
+        idx = torch.full((max(int(cu_B[-1]), 1),), -1, dtype=torch.int32, device="cuda")
+        pafu.pafu_select(torch.from_numpy(s).cuda(), shape, pol, idx)
+        got = idx.cpu().numpy()
+        for st in range(n):
+            want = oracle.select(s[cuT[st]:cuT[st + 1]], ns, nr, Bs[st])
+            assert cu_B[st + 1] - cu_B[st] == len(want)
+            assert np.array_equal(got[cu_B[st]:cu_B[st + 1]], want), (kind, ci, st)
+
+
+# ------------------------------------------------------------------------------- compact
+@pytest.mark.parametrize("w", SMALL + [wl.Workload("odd_dm", 7, 5, 8, (77, 9), (30, 9), 2, 3, (4, 4), 32)],
+                         ids=lambda w: "%s-dm%d" % (w.name, w.d_model))
+def test_compact_bit_exact(w):
+    d = wl.make_layer(w, tensors=("K", "V"))
+    rng = np.random.default_rng(3)
+    cuT = w.cu("T"); cuB = w.cu("B")
+    idx_np = np.concatenate([np.sort(rng.choice(w.T[s], size=cuB[s + 1] - cuB[s], replace=False))
+                             for s in range(w.n_streams)]).astype(np.int32)
+    SL = rng.standard_normal(int(cuT[-1])).astype(np.float32)
+    shape = pafu.Shape(w.n_heads, w.d_head, cuT, None)
+    pol = pafu.make_policy(w.n_sink, w.n_recent, list(w.budget), w.n_streams)
+    K, V = to_device_bf16(d["K"]), to_device_bf16(d["V"])
+    nB = int(cuB[-1])
+    Kc = torch.zeros((nB, w.n_heads, w.d_head), dtype=torch.bfloat16, device="cuda")
+    Vc = torch.zeros_like(Kc)
+    SLc = torch.zeros(nB, device="cuda")
+    pafu.pafu_compact(K, V, torch.from_numpy(SL).cuda(), torch.from_numpy(idx_np).cuda(), shape, pol,
+                      Kc, Vc, SLc)
+    for s in range(w.n_streams):
+        i = idx_np[cuB[s]:cuB[s + 1]]
+        assert np.array_equal(bf16_to_bits(Kc)[cuB[s]:cuB[s + 1]], oracle.compact(d["K"][cuT[s]:cuT[s + 1]], i))
+        assert np.array_equal(bf16_to_bits(Vc)[cuB[s]:cuB[s + 1]], oracle.compact(d["V"][cuT[s]:cuT[s + 1]], i))
+        assert np.array_equal(SLc.cpu().numpy()[cuB[s]:cuB[s + 1]], oracle.compact(SL[cuT[s]:cuT[s + 1]], i))
+    # inputs untouched
+    assert np.array_equal(bf16_to_bits(K), d["K"]) and np.array_equal(bf16_to_bits(V), d["V"])
+
+
+# ----------------------------------------------------------------------------- attention
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: "%s-d%d" % (w.name, w.d_head))
+def test_attention_matches_oracle_everywhere(w):
+    d = wl.make_layer(w)
+    L = Layer(w, d)
+    # retained cache = the oracle's own selection, so attention is tested on its own
+    sc = oracle_scores(w, d)
+    idx = oracle_select_streams(sc, w)
+    cuT, cuB = w.cu("T"), L.cu_B
+    Kc = np.concatenate([oracle.compact(d["K"][cuT[s]:cuT[s + 1]], idx[s]) for s in range(w.n_streams)])
+    Vc = np.concatenate([oracle.compact(d["V"][cuT[s]:cuT[s + 1]], idx[s]) for s in range(w.n_streams)])
+    L.Kc.copy_(to_device_bf16(Kc)); L.Vc.copy_(to_device_bf16(Vc))
+    L.O.fill_(float("nan")); L.LSE.fill_(float("nan"))
+    L.attn()
+    L.check_status()
+    got = wl.bf16_bits_to_f32(bf16_to_bits(L.O))
+    lse = L.LSE.cpu().numpy()
+    cuQ = w.cu("Lq")
+    for s, (O, Ls) in enumerate(oracle_attn_streams(w, d, Kc, Vc, cuB)):
+        close(got[cuQ[s]:cuQ[s + 1]], O, "attn O stream %d" % s)
+        close(lse[:, cuQ[s]:cuQ[s + 1]], Ls, "attn LSE stream %d" % s)
+
+
+def test_attention_segment_edge_cases():
+    # no retained cache / no chunk segment / one key / lengths around the tile sizes
+    rng = np.random.default_rng(9)
+    N, D = 2, 128
+    for (Lq, nB, chunk) in [(1, 0, True), (5, 1, False), (64, 64, True), (65, 127, True),
+                            (129, 128, False), (130, 257, True), (3, 0, False)]:
+        bits = lambda n: wl.f32_to_bf16_bits(rng.standard_normal((n, N, D)).astype(np.float32))
+        Q, Kc, Vc, Kq, Vq = bits(Lq), bits(nB), bits(nB), bits(Lq), bits(Lq)
+        shape = pafu.Shape(N, D, None, [0, Lq])
+        dv = lambda a: to_device_bf16(a) if a.shape[0] else torch.zeros((1, N, D), dtype=torch.bfloat16, device="cuda")
+        O = torch.full((Lq, N, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        LSE = torch.full((N, Lq), float("nan"), device="cuda")
+        ws = torch.zeros(max(pafu.pafu_workspace_bytes(shape), 256), dtype=torch.uint8, device="cuda")
+        pafu.pafu_chunk_attn(dv(Q), dv(Kc), dv(Vc), [0, nB], dv(Kq) if chunk else None,
+                             dv(Vq) if chunk else None, shape, 0.0, O, LSE, ws)
+        assert pafu.pafu_workspace_status(ws) == 0
+        want, wl_ = oracle.attention(Q, Kc, Vc, Kq if chunk else None, Vq if chunk else None)
+        got = wl.bf16_bits_to_f32(bf16_to_bits(O))
+        if nB == 0 and not chunk:
+            assert np.all(got == 0) and np.all(np.isneginf(LSE.cpu().numpy()))
+        else:
+            close(got, want, "edge O %s" % ((Lq, nB, chunk),))
+            close(LSE.cpu().numpy(), wl_, "edge LSE")
+
+
+# ---------------------------------------------------------------------------------- step
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: "%s-d%d" % (w.name, w.d_head))
+def test_step_equals_four_calls_and_oracle(w):
+    d = wl.make_layer(w)
+    A = Layer(w, d); B = Layer(w, d)
+    A.step(); A.check_status()
+    B.score(); B.select(); B.compact(); B.attn(); B.check_status()
+    for name in ("scores", "idx", "Kc", "Vc", "SLc", "O", "LSE"):
+        a, b = getattr(A, name), getattr(B, name)
+        n = {"scores": A.nT, "idx": A.nB, "Kc": A.nB, "Vc": A.nB, "SLc": A.nB}.get(name)
+        if n is not None:
+            a, b = a[:n], b[:n]
+        assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a,
+                           b.view(torch.int16) if b.dtype == torch.bfloat16 else b), name
+    # against the oracle: scores within tolerance; indices exact given the GPU's own fp32 scores;
+    # compacted K/V/SL byte-identical given those indices; attention within tolerance
+    gs = A.scores[: A.nT].cpu().numpy()
+    close(gs, oracle_scores(w, d), "step scores")
+    idx = oracle_select_streams(gs, w)
+    got_idx = A.idx[: A.nB].cpu().numpy()
+    cuT, cuB, cuQ = w.cu("T"), A.cu_B, w.cu("Lq")
+    Kc_bits, Vc_bits = bf16_to_bits(A.Kc)[: A.nB], bf16_to_bits(A.Vc)[: A.nB]
+    for s in range(w.n_streams):
+        assert np.array_equal(got_idx[cuB[s]:cuB[s + 1]], idx[s])
+        assert np.array_equal(Kc_bits[cuB[s]:cuB[s + 1]], oracle.compact(d["K"][cuT[s]:cuT[s + 1]], idx[s]))
+        assert np.array_equal(Vc_bits[cuB[s]:cuB[s + 1]], oracle.compact(d["V"][cuT[s]:cuT[s + 1]], idx[s]))
+        assert np.array_equal(A.SLc.cpu().numpy()[cuB[s]:cuB[s + 1]], gs[cuT[s]:cuT[s + 1]][idx[s]])
+    got = wl.bf16_bits_to_f32(bf16_to_bits(A.O))
+    for s, (O, Ls) in enumerate(oracle_attn_streams(w, d, Kc_bits, Vc_bits, cuB)):
+        close(got[cuQ[s]:cuQ[s + 1]], O, "step O")
+
+
+def test_step_host_matches_device_step():
+    w = wl.small_ragged(2, 128)
+    d = wl.make_layer(w)
+    A = Layer(w, d)
+    A.step(); A.check_status()
+    host = {k: torch.from_numpy(v.view(np.int16)).pin_memory() for k, v in d.items()}
+    scores = torch.empty(A.nT, dtype=torch.float32).pin_memory()
+    idx = torch.empty(A.nB, dtype=torch.int32).pin_memory()
+    O = torch.empty((A.nQ, w.n_heads, w.d_head), dtype=torch.int16).pin_memory()
+    head = pafu.Head(host["w1"], host["b1"], host["w2"], host["b2"], w.act, w.final)
+    arena = torch.empty(pafu.pafu_step_host_arena_bytes(A.shape, A.policy, head), dtype=torch.uint8, device="cuda")
+    args = pafu.step_args(A.shape, head, A.policy, host["K"], host["V"], host["Q"], host["Kq"], host["Vq"],
+                          0.0, scores, idx, None, None, None, O, None, None)
+    pafu.pafu_step_host(args, arena)
+    assert torch.equal(scores, A.scores[: A.nT].cpu())
+    assert torch.equal(idx, A.idx[: A.nB].cpu())
+    assert torch.equal(O, A.O.view(torch.int16).cpu())
+
+
+# ---------------------------------------------------------------------- full-size configs
+def _full_size_check(w, n_rows=256, seed=0):
+    d = wl.make_layer(w, seed=seed)
+    L = Layer(w, d)
+    L.step(); L.check_status()
+    torch.cuda.synchronize()
+    gs = L.scores[: L.nT].cpu().numpy()
+    close(gs, oracle_scores(w, d), "scores")
+    idx = oracle_select_streams(gs, w)
+    got_idx = L.idx[: L.nB].cpu().numpy()
+    cuT, cuB, cuQ = w.cu("T"), L.cu_B, w.cu("Lq")
+    Kc_bits, Vc_bits = bf16_to_bits(L.Kc)[: L.nB], bf16_to_bits(L.Vc)[: L.nB]
+    rows = []
+    for s in range(w.n_streams):
+        assert np.array_equal(got_idx[cuB[s]:cuB[s + 1]], idx[s])
+        assert np.array_equal(Kc_bits[cuB[s]:cuB[s + 1]], oracle.compact(d["K"][cuT[s]:cuT[s + 1]], idx[s]))
+        assert np.array_equal(Vc_bits[cuB[s]:cuB[s + 1]], oracle.compact(d["V"][cuT[s]:cuT[s + 1]], idx[s]))
+        r = set(wl.sample_rows(w.Lq[s], n_rows, seed=seed, tag=s).tolist())
+        last_tile = (w.Lq[s] // 128) * 128          # rows of the partial last tile
+        r |= set(range(last_tile, w.Lq[s])[:: max(1, (w.Lq[s] - last_tile) // 16)])
+        rows.append(np.array(sorted(r), dtype=np.int64))
+    got = wl.bf16_bits_to_f32(bf16_to_bits(L.O))
+    lse = L.LSE.cpu().numpy()
+    for s, (O, Ls) in enumerate(oracle_attn_streams(w, d, Kc_bits, Vc_bits, cuB, rows)):
+        close(got[cuQ[s]:cuQ[s + 1]][rows[s]], O, "O stream %d" % s)
+        close(lse[:, cuQ[s]:cuQ[s + 1]][:, rows[s]], Ls, "LSE stream %d" % s)
+
+
+def test_full_size_wan13b_layer():
+    _full_size_check(wl.wan13b_layer())
+
+
+def test_full_size_paper_native_point():
+    _full_size_check(wl.paper_native(), n_rows=96)
