@@ -141,11 +141,9 @@ pafu_status pafu_score(const pafu_head* head, const uint16_t* X, int64_t n_token
     if (ldx < head->d_in || ldx % 8 != 0) return PAFU_ERR_INVALID_ARG;
     if (!aligned16(X) || !aligned16(scores)) return PAFU_ERR_MISALIGNED;
     const size_t need = kWsHeaderBytes + score_workspace_bytes(*head);
-    if (need > kWsHeaderBytes) {
-        if (ws == nullptr) return PAFU_ERR_INVALID_ARG;
-        if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
-        if (ws_bytes < need) return PAFU_ERR_WORKSPACE_TOO_SMALL;
-    }
+    if (ws == nullptr) return PAFU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
+    if (ws_bytes < need) return PAFU_ERR_WORKSPACE_TOO_SMALL;
     return launch_score(*head, X, n_tokens, ldx, scores, ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
@@ -208,11 +206,9 @@ pafu_status pafu_chunk_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_
     if (!aligned16(Q) || !aligned16(O) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(Kq) ||
         !aligned16(Vq) || !aligned16(LSE)) return PAFU_ERR_MISALIGNED;
     const size_t need = kWsHeaderBytes + attn_workspace_bytes(st, shape->n_heads, shape->d_head);
-    if (need > kWsHeaderBytes) {
-        if (ws == nullptr) return PAFU_ERR_INVALID_ARG;
-        if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
-        if (ws_bytes < need) return PAFU_ERR_WORKSPACE_TOO_SMALL;
-    }
+    if (ws == nullptr) return PAFU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
+    if (ws_bytes < need) return PAFU_ERR_WORKSPACE_TOO_SMALL;
     if (scale == 0.f) scale = 1.0f / sqrtf((float)shape->d_head);
     return launch_attn(Q, Kc, Vc, Kq, Vq, st, shape->n_heads, shape->d_head, scale, O, LSE, ws, ws_bytes,
                        static_cast<cudaStream_t>(stream));
@@ -254,11 +250,9 @@ static pafu_status step_impl(const pafu_step_args* a, void* const* ev, void* str
         if (!aligned16(p)) return PAFU_ERR_MISALIGNED;
     if (nB > 0 && (a->Kc == a->K || a->Vc == a->V || a->Kc == a->V || a->Vc == a->K)) return PAFU_ERR_INVALID_ARG;
     const size_t need = pafu_workspace_bytes(&a->shape, a->policy, a->head);
-    if (need > kWsHeaderBytes) {
-        if (a->ws == nullptr) return PAFU_ERR_INVALID_ARG;
-        if ((reinterpret_cast<uintptr_t>(a->ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
-        if (a->ws_bytes < need) return PAFU_ERR_WORKSPACE_TOO_SMALL;
-    }
+    if (a->ws == nullptr) return PAFU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(a->ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
+    if (a->ws_bytes < need) return PAFU_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     auto mark = [&](int i) -> bool {
         return ev == nullptr || cudaEventRecord(static_cast<cudaEvent_t>(ev[i]), cs) == cudaSuccess;

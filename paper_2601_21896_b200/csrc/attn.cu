@@ -1,6 +1,7 @@
 // Chunk attention launcher: picks the kernel for the shape.
 #include "common.cuh"
 #include "attn_mma.cuh"
+#include "attn_tc.cuh"
 
 namespace pafu {
 
@@ -9,7 +10,10 @@ size_t attn_workspace_bytes(const StreamTable&, int32_t, int32_t) { return 0; }
 pafu_status launch_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
                         const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
                         int32_t n_heads, int32_t d_head, float scale, uint16_t* O, float* LSE,
-                        void*, size_t, cudaStream_t stream) {
+                        void* ws, size_t, cudaStream_t stream) {
+    if (d_head == attn_tc::kD)
+        return attn_tc::launch(Q, Kc, Vc, Kq, Vq, st, n_heads, scale, O, LSE,
+                               reinterpret_cast<int*>(ws) + kStatusWordTimeout, stream);
     return attn_mma::launch(Q, Kc, Vc, Kq, Vq, st, n_heads, d_head, scale, O, LSE, stream);
 }
 
