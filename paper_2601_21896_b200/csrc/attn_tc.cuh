@@ -3,13 +3,22 @@
 //   o_i = sum_j softmax_j(scale q_i.k_j) v_j,  j over [retained cache ; chunk tokens]
 //   (Sec. 3.2 for the operator; Eq. 2 / Eq. 7 for the key range)
 //
-// One CTA works on 256 query rows of one head as two 128-row "slots" that share every K/V
-// tile, so each tile is fetched once per 256 rows.  Warp roles:
+// Work decomposition.  An "item" is 256 query rows of one head of one stream, handled as two
+// 128-row "slots" that share every K/V tile (each tile is fetched once per 256 rows).  The
+// grid is persistent: one CTA per SM.  All items' key tiles are laid end to end and cut into
+// equal contiguous shares, one per CTA (cost of a tile = number of live slots), so every SM
+// gets the same amount of tensor work whatever the item count.  A CTA whose share covers only
+// part of an item's keys writes an unnormalised partial (O, running max, row sum) to the
+// workspace; a second small kernel merges the partials of each split item in key order, which
+// keeps the result deterministic.
+//
+// Warp roles inside a CTA (384 threads):
 //   warps 0-3  softmax of slot 0 (thread = query row = TMEM lane)
 //   warps 4-7  softmax of slot 1
 //   warp  8    MMA issuer: S = Q K^T (both operands in shared memory) and O += P V
 //              (P read from tensor memory, V from shared memory, MN-major)
-//   warp  9    TMA loader: Q tiles once, then K/V tiles through a 5-stage ring
+//   warp  9    TMA loader: Q tiles per item, K/V tiles through a 5-stage ring that runs
+//              ahead across item boundaries
 //   warps 10-11 idle (they complete the third warpgroup so registers can be re-balanced)
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; the bf16 P tile
 // overwrites the first 64 columns of its S tile.  While one slot runs its softmax the tensor
@@ -35,11 +44,21 @@ constexpr int kD = 128;
 constexpr int kBM = 128;            // query rows per slot
 constexpr int kBN = 128;            // keys per tile
 constexpr int kStages = 5;          // K/V ring depth (each stage one 128 x 128 bf16 tile)
-constexpr int kThreads = 384;           // 3 warpgroups: softmax 0, softmax 1, {MMA, loader, 2 idle}
+constexpr int kThreads = 384;       // 3 warpgroups: softmax 0, softmax 1, {MMA, loader, 2 idle}
 constexpr int kTileBytes = kBN * kD * 2;      // 32 KiB
 constexpr int kHalfBytes = kTileBytes / 2;    // one [128 rows x 64 cols] swizzled half
 constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 1024 /*align*/ + 256 /*barriers*/;
 constexpr float kRescaleThresholdLog2 = 8.0f;
+// Register re-balancing.  With 384 threads the kernel launches with 168 registers per thread.
+// setmaxnreg.inc blocks until the registers exist, so what the third warpgroup gives up must
+// cover what the two softmax warpgroups take: (168 - kRegsLow) * 128 >= (kRegsHigh - 168) * 256.
+constexpr int kRegsLaunch = 168, kRegsLow = 80, kRegsHigh = 208;
+static_assert((kRegsLaunch - kRegsLow) * 128 >= (kRegsHigh - kRegsLaunch) * 256,
+              "setmaxnreg.inc would wait forever");
+constexpr int kMaxGrid = 256;
+// one partial: O [256][128] fp32, then m [256], then l [256]
+constexpr int kPieceFloats = 2 * kBM * kD + 2 * 2 * kBM;
+constexpr size_t kPieceBytes = (size_t)kPieceFloats * 4;
 
 struct Params {
     StreamTable st;
@@ -49,36 +68,87 @@ struct Params {
     uint16_t* O;
     float* LSE;
     int* status;        // workspace status word (device)
+    float* pieces;      // [gridDim][2][kPieceFloats]
     int64_t total_Lq;
+    int64_t total_cost;
 };
 
-struct Item {            // one CTA's work: 256 query rows of one head of one stream
-    int stream, head;
+// A contiguous run of key tiles [t0, t1) of one item, as seen by one CTA.
+struct Seg {
+    int stream, head, n_slots;
     int64_t q0;          // first query row (stream-local)
     int64_t Lq, nB, nC;  // stream's query rows, retained keys, chunk keys
-    int nt1, nt2;        // key tiles in each segment
+    int nt1, nt, t0, t1; // tiles in the retained segment, tiles in total, this run
+    int piece;           // -1: whole item (final output); 0: continues an item begun by an
+                         // earlier CTA; 1: begins an item that a later CTA continues
 };
 
-__device__ __forceinline__ Item decode_item(const Params& p, int64_t item) {
-    Item it;
-    int s = 0;
-    for (;; ++s) {
-        const int64_t lq = p.st.cu_Lq[s + 1] - p.st.cu_Lq[s];
-        const int64_t n = ((lq + 2 * kBM - 1) / (2 * kBM)) * p.n_heads;
-        if (item < n) break;
-        item -= n;
-    }
-    it.stream = s;
-    it.Lq = p.st.cu_Lq[s + 1] - p.st.cu_Lq[s];
-    const int64_t nqp = (it.Lq + 2 * kBM - 1) / (2 * kBM);
-    it.head = (int)(item / nqp);
-    it.q0 = (item % nqp) * (2 * kBM);
-    it.nB = p.st.cu_B[s + 1] - p.st.cu_B[s];
-    it.nC = p.has_chunk ? it.Lq : 0;
-    it.nt1 = (int)((it.nB + kBN - 1) / kBN);
-    it.nt2 = (int)((it.nC + kBN - 1) / kBN);
-    return it;
+struct StreamCost {
+    int64_t nqp, nt, head_cost;
+    int tail_slots;
+};
+
+__host__ __device__ inline StreamCost stream_cost(const StreamTable& st, int s, int has_chunk) {
+    StreamCost c;
+    const int64_t lq = st.cu_Lq[s + 1] - st.cu_Lq[s];
+    const int64_t nB = st.cu_B[s + 1] - st.cu_B[s];
+    c.nqp = (lq + 2 * kBM - 1) / (2 * kBM);
+    c.tail_slots = (lq - (c.nqp - 1) * 2 * kBM > kBM) ? 2 : 1;
+    c.nt = (nB + kBN - 1) / kBN + (has_chunk ? (lq + kBN - 1) / kBN : 0);
+    c.head_cost = (lq > 0) ? c.nt * (2 * (c.nqp - 1) + c.tail_slots) : 0;
+    return c;
 }
+
+__host__ __device__ inline int64_t total_cost(const StreamTable& st, int n_heads, int has_chunk) {
+    int64_t t = 0;
+    for (int s = 0; s < st.n_streams; ++s) t += stream_cost(st, s, has_chunk).head_cost * n_heads;
+    return t;
+}
+
+// Walks the runs of one CTA's share [c0, c1) of the cost line.  Only the first run of a CTA
+// can start inside an item (t0 > 0) and only its last run can stop inside one (t1 < nt).
+struct SegIter {
+    int64_t cur, c1;
+    __device__ SegIter(const Params& p, int cta, int n_cta) {
+        cur = p.total_cost * cta / n_cta;
+        c1 = p.total_cost * (cta + 1) / n_cta;
+    }
+    __device__ bool next(const Params& p, Seg& g) {
+        while (cur < c1) {
+            int64_t c = cur;
+            int s = 0;
+            StreamCost sc;
+            for (;; ++s) {
+                sc = stream_cost(p.st, s, p.has_chunk);
+                const int64_t tot = sc.head_cost * p.n_heads;
+                if (c < tot) break;
+                c -= tot;
+            }
+            g.stream = s;
+            g.head = (int)(c / sc.head_cost);
+            const int64_t r = c % sc.head_cost;
+            const int64_t full = sc.nt * 2 * (sc.nqp - 1);
+            int64_t qp, rr;
+            if (r < full) { qp = r / (2 * sc.nt); rr = r % (2 * sc.nt); g.n_slots = 2; }
+            else { qp = sc.nqp - 1; rr = r - full; g.n_slots = sc.tail_slots; }
+            g.q0 = qp * 2 * kBM;
+            g.Lq = p.st.cu_Lq[s + 1] - p.st.cu_Lq[s];
+            g.nB = p.st.cu_B[s + 1] - p.st.cu_B[s];
+            g.nC = p.has_chunk ? g.Lq : 0;
+            g.nt1 = (int)((g.nB + kBN - 1) / kBN);
+            g.nt = (int)sc.nt;
+            const int64_t item_start = cur - rr, item_end = item_start + sc.nt * g.n_slots;
+            g.t0 = (int)(rr / g.n_slots);
+            if (c1 >= item_end) { g.t1 = g.nt; cur = item_end; }
+            else { g.t1 = (int)((c1 - item_start) / g.n_slots); cur = c1; }
+            if (g.t1 > g.t0) {
+                g.piece = (g.t0 == 0 && g.t1 == g.nt) ? -1 : (g.t0 > 0 ? 0 : 1);
+                return true;
+            }
+        }
+        return false;
+    }
+};
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -100,25 +170,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     const uint32_t sQ = smem_u32(smem);                       // 2 slots x 32 KiB
     const uint32_t sKV = sQ + 2 * kTileBytes;                 // ring
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kTileBytes + kStages * kTileBytes);
-    // barrier map
     const uint32_t bar0 = smem_u32(bars);
     auto q_full = [&](int s) { return bar0 + 8 * (0 + s); };
-    auto s_full = [&](int s) { return bar0 + 8 * (2 + s); };
-    auto p_full = [&](int s) { return bar0 + 8 * (4 + s); };
-    auto o_done = [&](int s) { return bar0 + 8 * (6 + s); };
-    auto kv_full = [&](int st) { return bar0 + 8 * (8 + st); };
-    auto kv_empty = [&](int st) { return bar0 + 8 * (8 + kStages + st); };
+    auto q_empty = [&](int s) { return bar0 + 8 * (2 + s); };
+    auto s_full = [&](int s) { return bar0 + 8 * (4 + s); };
+    auto p_full = [&](int s) { return bar0 + 8 * (6 + s); };
+    auto o_done = [&](int s) { return bar0 + 8 * (8 + s); };
+    auto kv_full = [&](int st) { return bar0 + 8 * (10 + st); };
+    auto kv_empty = [&](int st) { return bar0 + 8 * (10 + kStages + st); };
     __shared__ uint32_t tmem_base_sh;
     __shared__ volatile int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const Item it = decode_item(p, blockIdx.x);
-    const int ntiles = it.nt1 + it.nt2;
-    const int n_slots = (it.q0 + kBM < it.Lq) ? 2 : 1;
 
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
-            mbar_init(q_full(s), 1); mbar_init(s_full(s), 1); mbar_init(p_full(s), kBM); mbar_init(o_done(s), 1);
+            mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1); mbar_init(s_full(s), 1);
+            mbar_init(p_full(s), kBM); mbar_init(o_done(s), 1);
         }
         for (int st = 0; st < kStages; ++st) { mbar_init(kv_full(st), 1); mbar_init(kv_empty(st), 1); }
         abort_flag = 0;
@@ -138,38 +206,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     if (warp >= 8) {
     // register budget: this warpgroup gives registers up, the softmax warpgroups (which hold a
     // whole S row per thread) take them
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLow));
     if (warp == 9) {
         // ------------------------------------------------------------------ TMA loader
         if (elect_one()) {
             prefetch_tmap(&mQ); prefetch_tmap(&mKc); prefetch_tmap(&mVc);
             if (p.has_chunk) { prefetch_tmap(&mKq); prefetch_tmap(&mVq); }
-            const int qrow = (int)(p.st.cu_Lq[it.stream] + it.q0);
-            for (int s = 0; s < n_slots; ++s) {
-                mbar_arrive_expect_tx(q_full(s), kTileBytes);
-                tma_load_3d(sQ + s * kTileBytes, &mQ, q_full(s), 0, it.head, qrow + s * kBM);
-                tma_load_3d(sQ + s * kTileBytes + kHalfBytes, &mQ, q_full(s), 64, it.head, qrow + s * kBM);
-            }
-            int ring = 0;
+            SegIter iter(p, blockIdx.x, gridDim.x);
+            Seg g;
+            uint32_t ring = 0, qcnt[2] = {0, 0};
             bool ok = true;
-            for (int j = 0; j < ntiles && ok; ++j) {
-                const bool seg2 = j >= it.nt1;
-                const int row = seg2 ? (int)(p.st.cu_Lq[it.stream] + (int64_t)(j - it.nt1) * kBN)
-                                     : (int)(p.st.cu_B[it.stream] + (int64_t)j * kBN);
-                for (int kv = 0; kv < 2 && ok; ++kv, ++ring) {
-                    const int st = ring % kStages;
-                    const uint32_t ph = (uint32_t)(ring / kStages) & 1u;
-                    if (abort_flag || !mbar_wait(kv_empty(st), ph ^ 1u)) { fail(101); ok = false; break; }
-                    const CUtensorMap* m = seg2 ? (kv ? &mVq : &mKq) : (kv ? &mVc : &mKc);
-                    mbar_arrive_expect_tx(kv_full(st), kTileBytes);
-                    tma_load_3d(sKV + st * kTileBytes, m, kv_full(st), 0, it.head, row);
-                    tma_load_3d(sKV + st * kTileBytes + kHalfBytes, m, kv_full(st), 64, it.head, row);
+            while (ok && iter.next(p, g)) {
+                const int qrow = (int)(p.st.cu_Lq[g.stream] + g.q0);
+                for (int s = 0; s < g.n_slots && ok; ++s) {
+                    if (abort_flag || !mbar_wait(q_empty(s), (qcnt[s] & 1u) ^ 1u)) { fail(100); ok = false; break; }
+                    ++qcnt[s];
+                    mbar_arrive_expect_tx(q_full(s), kTileBytes);
+                    tma_load_3d(sQ + s * kTileBytes, &mQ, q_full(s), 0, g.head, qrow + s * kBM);
+                    tma_load_3d(sQ + s * kTileBytes + kHalfBytes, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
+                }
+                for (int j = g.t0; j < g.t1 && ok; ++j) {
+                    const bool seg2 = j >= g.nt1;
+                    const int row = seg2 ? (int)(p.st.cu_Lq[g.stream] + (int64_t)(j - g.nt1) * kBN)
+                                         : (int)(p.st.cu_B[g.stream] + (int64_t)j * kBN);
+                    for (int kv = 0; kv < 2; ++kv, ++ring) {
+                        const int st = ring % kStages;
+                        const uint32_t ph = (ring / kStages) & 1u;
+                        if (abort_flag || !mbar_wait(kv_empty(st), ph ^ 1u)) { fail(101); ok = false; break; }
+                        const CUtensorMap* m = seg2 ? (kv ? &mVq : &mKq) : (kv ? &mVc : &mKc);
+                        mbar_arrive_expect_tx(kv_full(st), kTileBytes);
+                        tma_load_3d(sKV + st * kTileBytes, m, kv_full(st), 0, g.head, row);
+                        tma_load_3d(sKV + st * kTileBytes + kHalfBytes, m, kv_full(st), 64, g.head, row);
+                    }
                 }
             }
             if (!ok) {
                 // let copies already in flight land before the CTA exits
-                for (int r = max(0, ring - kStages); r < ring; ++r)
-                    mbar_wait(kv_full(r % kStages), (uint32_t)(r / kStages) & 1u);
+                for (uint32_t r = ring > (uint32_t)kStages ? ring - kStages : 0; r < ring; ++r)
+                    mbar_wait(kv_full(r % kStages), (r / kStages) & 1u);
             }
         }
         __syncwarp();
@@ -200,32 +274,40 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 if (!ok) return;
                 if (abort_flag || !mbar_wait(bar, ph)) { fail(code); ok = false; }
             };
-            for (int s = 0; s < n_slots; ++s) wait(q_full(s), 0, 201);
-            if (ntiles > 0) {
-                wait(kv_full(0), 0, 202);
-                if (ok) {
-                    tc_fence_after_sync();
-                    for (int s = 0; s < n_slots; ++s) { issue_qk(s, 0); umma_commit(s_full(s)); }
-                    umma_commit(kv_empty(0));
-                }
-            }
-            for (int j = 0; j < ntiles && ok; ++j) {
-                const int rv = 2 * j + 1, rk = 2 * j + 2;          // ring slots of V_j and K_{j+1}
-                const int stv = rv % kStages, stk = rk % kStages;
-                wait(kv_full(stv), (uint32_t)(rv / kStages) & 1u, 203);
-                const bool more = j + 1 < ntiles;
-                if (more) wait(kv_full(stk), (uint32_t)(rk / kStages) & 1u, 204);
-                for (int s = 0; s < n_slots && ok; ++s) {
-                    wait(p_full(s), (uint32_t)j & 1u, 205);
+            SegIter iter(p, blockIdx.x, gridDim.x);
+            Seg g;
+            uint32_t ring = 0, qcnt[2] = {0, 0}, pcnt[2] = {0, 0};
+            while (ok && iter.next(p, g)) {
+                for (int s = 0; s < g.n_slots; ++s) { wait(q_full(s), qcnt[s] & 1u, 201); ++qcnt[s]; }
+                {   // S(t0) for every live slot
+                    const int st = ring % kStages;
+                    wait(kv_full(st), (ring / kStages) & 1u, 202);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    issue_pv(s, stv, j == 0);
-                    if (more) { issue_qk(s, stk); umma_commit(s_full(s)); }
-                    else umma_commit(o_done(s));
+                    for (int s = 0; s < g.n_slots; ++s) { issue_qk(s, st); umma_commit(s_full(s)); }
+                    umma_commit(kv_empty(st));
+                    ++ring;
                 }
-                if (ok) {
-                    umma_commit(kv_empty(stv));
-                    if (more) umma_commit(kv_empty(stk));
+                for (int j = g.t0; j < g.t1 && ok; ++j) {
+                    const bool more = j + 1 < g.t1;
+                    const uint32_t rv = ring, rk = ring + 1;           // V_j and K_{j+1}
+                    const int stv = rv % kStages, stk = rk % kStages;
+                    wait(kv_full(stv), (rv / kStages) & 1u, 203);
+                    if (more) wait(kv_full(stk), (rk / kStages) & 1u, 204);
+                    for (int s = 0; s < g.n_slots && ok; ++s) {
+                        wait(p_full(s), pcnt[s] & 1u, 205);
+                        if (!ok) break;
+                        ++pcnt[s];
+                        tc_fence_after_sync();
+                        issue_pv(s, stv, j == g.t0);
+                        if (more) { issue_qk(s, stk); umma_commit(s_full(s)); }
+                        else { umma_commit(o_done(s)); umma_commit(q_empty(s)); }
+                    }
+                    if (ok) {
+                        umma_commit(kv_empty(stv));
+                        if (more) umma_commit(kv_empty(stk));
+                    }
+                    ring += more ? 2 : 1;
                 }
             }
         }
@@ -233,20 +315,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     }
     } else {
         // ------------------------------------------------------------------ softmax warps
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsHigh));
         const int slot = warp >> 2;
         const int row_in_slot = tid & 127;
         const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
         const uint32_t tS = tmem + slot * kBN + lane_base;
         const uint32_t tO = tmem + 256 + slot * kD + lane_base;
         const float sl2 = p.scale * 1.4426950408889634f;
-        float m_used = -INFINITY, l_sum = 0.f;
-        bool ok = slot < n_slots;
-        if (ok) {
-            for (int j = 0; j < ntiles; ++j) {
+        SegIter iter(p, blockIdx.x, gridDim.x);
+        Seg g;
+        uint32_t scnt = 0, ocnt = 0;
+        bool ok = true;
+        while (ok && iter.next(p, g)) {
+            if (slot >= g.n_slots) continue;
+            float m_used = -INFINITY, l_sum = 0.f;
+            for (int j = g.t0; j < g.t1; ++j) {
                 {
-                    const bool w = mbar_wait(s_full(slot), (uint32_t)j & 1u) && !abort_flag;
+                    const bool w = mbar_wait(s_full(slot), scnt & 1u) && !abort_flag;
                     if (!__all_sync(0xffffffffu, w)) { fail(301); ok = false; break; }   // warp-uniform
+                    ++scnt;
                 }
                 tc_fence_after_sync();
                 uint32_t sr[128];
@@ -256,8 +343,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 PAFU_TMEM_LD_X32(tS + 96, sr + 96);
                 tmem_wait_ld();
                 // ragged end of a key segment
-                const bool seg2 = j >= it.nt1;
-                const int64_t left = (seg2 ? it.nC - (int64_t)(j - it.nt1) * kBN : it.nB - (int64_t)j * kBN);
+                const bool seg2 = j >= g.nt1;
+                const int64_t left = (seg2 ? g.nC - (int64_t)(j - g.nt1) * kBN : g.nB - (int64_t)j * kBN);
                 if (left < kBN) {
 #pragma unroll
                     for (int c = 0; c < 128; ++c)
@@ -266,7 +353,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 float mx = __uint_as_float(sr[0]);
 #pragma unroll
                 for (int c = 1; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
-                if (j == 0) {
+                if (j == g.t0) {
                     m_used = mx;
                 } else if (__any_sync(0xffffffffu, (mx - m_used) * sl2 > kRescaleThresholdLog2)) {
                     // the whole warp rescales together (TMEM accesses are warp-collective);
@@ -304,28 +391,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 tc_fence_before_sync();
                 mbar_arrive(p_full(slot));
             }
-        }
-        if (ok) {
-            const int64_t row = it.q0 + slot * kBM + row_in_slot;
-            if (ntiles > 0) {
-                const bool w = mbar_wait(o_done(slot), 0) && !abort_flag;
-                if (!__all_sync(0xffffffffu, w)) { fail(302); ok = false; }
-                tc_fence_after_sync();
+            if (!ok) break;
+            {
+                const bool w = mbar_wait(o_done(slot), ocnt & 1u) && !abort_flag;
+                if (!__all_sync(0xffffffffu, w)) { fail(302); ok = false; break; }
+                ++ocnt;
             }
-            if (ok) {
+            tc_fence_after_sync();
+            const int64_t row = g.q0 + slot * kBM + row_in_slot;
+            if (g.piece < 0) {
+                // whole item: normalise and store bf16
                 const float inv = (l_sum > 0.f) ? 1.0f / l_sum : 0.f;
-                uint16_t* dst = p.O + ((p.st.cu_Lq[it.stream] + row) * p.n_heads + it.head) * kD;
+                uint16_t* dst = p.O + ((p.st.cu_Lq[g.stream] + row) * p.n_heads + g.head) * kD;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t orr[32];
-                    if (ntiles > 0) {
-                        PAFU_TMEM_LD_X32(tO + c * 32, orr);
-                        tmem_wait_ld();
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) orr[i] = 0u;
-                    }
-                    if (row < it.Lq) {
+                    PAFU_TMEM_LD_X32(tO + c * 32, orr);
+                    tmem_wait_ld();
+                    if (row < g.Lq) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             uint4 v;
@@ -337,9 +420,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                         }
                     }
                 }
-                if (p.LSE != nullptr && row < it.Lq)
-                    p.LSE[(int64_t)it.head * p.total_Lq + p.st.cu_Lq[it.stream] + row] =
+                if (p.LSE != nullptr && row < g.Lq)
+                    p.LSE[(int64_t)g.head * p.total_Lq + p.st.cu_Lq[g.stream] + row] =
                         (l_sum > 0.f) ? m_used * p.scale + logf(l_sum) : -INFINITY;
+            } else {
+                // part of an item: unnormalised fp32 partial for the merge kernel
+                float* piece = p.pieces + ((size_t)blockIdx.x * 2 + g.piece) * kPieceFloats;
+                const int prow = slot * kBM + row_in_slot;
+                float4* dst = reinterpret_cast<float4*>(piece + (size_t)prow * kD);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t orr[32];
+                    PAFU_TMEM_LD_X32(tO + c * 32, orr);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        dst[c * 8 + q] = make_float4(__uint_as_float(orr[4 * q]), __uint_as_float(orr[4 * q + 1]),
+                                                     __uint_as_float(orr[4 * q + 2]), __uint_as_float(orr[4 * q + 3]));
+                }
+                piece[2 * kBM * kD + prow] = m_used;
+                piece[2 * kBM * kD + 2 * kBM + prow] = l_sum;
             }
         }
     }
@@ -348,38 +448,135 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
+// Merges the partials of every item that was split across CTAs.  Block b owns the item that
+// CTA b of the main kernel began (its last run, stored as piece 1) and adds the following
+// CTAs' continuation pieces (their first run, piece 0) in key order.
+__global__ void __launch_bounds__(256)
+attn_tc_merge_kernel(const __grid_constant__ Params p, int n_cta) {
+    __shared__ int piece_cta[kMaxGrid];
+    __shared__ int n_pieces_sh;
+    const int b = blockIdx.x;
+    Seg g, last;
+    bool have = false;
+    {
+        SegIter iter(p, b, n_cta);
+        while (iter.next(p, g)) { last = g; have = true; }
+    }
+    if (!have || last.piece != 1) return;      // block-uniform
+    if (threadIdx.x == 0) {
+        int n = 0, t = last.t1;
+        piece_cta[n++] = b;
+        for (int c = b + 1; c < n_cta && t < last.nt; ++c) {
+            SegIter iter(p, c, n_cta);
+            if (!iter.next(p, g)) continue;    // an empty share holds no piece
+            t = g.t1;
+            piece_cta[n++] = c;
+        }
+        n_pieces_sh = n;
+    }
+    __syncthreads();
+    const int n_pieces = n_pieces_sh;
+    const float sl2 = p.scale * 1.4426950408889634f;
+    const int lane = threadIdx.x & 31, sub = threadIdx.x >> 5;   // 8 rows per pass, 32 float4 per row
+    const int n_rows = last.n_slots * kBM;
+    for (int r = sub; r < n_rows; r += 8) {
+        const int64_t row = last.q0 + r;
+        if (row >= last.Lq) break;
+        float M = -INFINITY;
+        for (int i = 0; i < n_pieces; ++i) {
+            const float* piece = p.pieces + ((size_t)piece_cta[i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
+            M = fmaxf(M, piece[2 * kBM * kD + r]);
+        }
+        float L = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < n_pieces; ++i) {
+            const float* piece = p.pieces + ((size_t)piece_cta[i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
+            const float w = fast_exp2((piece[2 * kBM * kD + r] - M) * sl2);
+            L += w * piece[2 * kBM * kD + 2 * kBM + r];
+            const float4 v = reinterpret_cast<const float4*>(piece + (size_t)r * kD)[lane];
+            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+        }
+        const float inv = (L > 0.f) ? 1.0f / L : 0.f;
+        uint16_t* dst = p.O + ((p.st.cu_Lq[last.stream] + row) * p.n_heads + last.head) * kD + lane * 4;
+        uint2 o;
+        o.x = pack_bf16(acc.x * inv, acc.y * inv);
+        o.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(dst) = o;
+        if (p.LSE != nullptr && lane == 0)
+            p.LSE[(int64_t)last.head * p.total_Lq + p.st.cu_Lq[last.stream] + row] =
+                (L > 0.f) ? M * p.scale + logf(L) : -INFINITY;
+    }
+}
+
+inline int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v < kMaxGrid ? v : kMaxGrid;
+        else
+            return 148;      // no device visible (sizing queries on a build host)
+    }
+    return n;
+}
+
+inline int grid_for(int64_t cost) {
+    const int sms = sm_count();
+    return (int)(cost < sms ? cost : sms);
+}
+
+// True when every stream with queries has at least one key (the cost line has no entry for a
+// key-less item).
+inline bool supports(const StreamTable& st, bool has_chunk) {
+    for (int s = 0; s < st.n_streams; ++s) {
+        const int64_t lq = st.cu_Lq[s + 1] - st.cu_Lq[s], nB = st.cu_B[s + 1] - st.cu_B[s];
+        if (lq > 0 && nB == 0 && !has_chunk) return false;
+    }
+    return true;
+}
+
+// Scratch for the partials: one pair per CTA.
+inline size_t workspace_bytes() { return (size_t)sm_count() * 2 * kPieceBytes; }
+
 // Tensor maps are rebuilt per call (a few microseconds of host work); nothing is cached, so
 // the library stays stateless.
 inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
                           const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
                           int32_t n_heads, float scale, uint16_t* O, float* LSE, int* status,
-                          cudaStream_t stream) {
+                          float* pieces, cudaStream_t stream) {
     const int n = st.n_streams;
     const int64_t nQ = st.cu_Lq[n], nB = st.cu_B[n];
-    int64_t items = 0;
-    for (int s = 0; s < n; ++s) items += ((st.cu_Lq[s + 1] - st.cu_Lq[s] + 2 * kBM - 1) / (2 * kBM)) * n_heads;
-    if (items == 0) return PAFU_OK;
+    const int has_chunk = Kq != nullptr;
+    const int64_t cost = total_cost(st, n_heads, has_chunk);
+    if (cost == 0) return PAFU_OK;
     CUtensorMap mQ, mKc, mVc, mKq, mVq;
     if (!TmapEncoder::token_tensor(&mQ, Q, (uint64_t)nQ, n_heads, kD, kBM)) return PAFU_ERR_CUDA;
     if (nB > 0) {
         if (!TmapEncoder::token_tensor(&mKc, Kc, (uint64_t)nB, n_heads, kD, kBN) ||
             !TmapEncoder::token_tensor(&mVc, Vc, (uint64_t)nB, n_heads, kD, kBN)) return PAFU_ERR_CUDA;
     } else { mKc = mQ; mVc = mQ; }
-    if (Kq != nullptr) {
+    if (has_chunk) {
         if (!TmapEncoder::token_tensor(&mKq, Kq, (uint64_t)nQ, n_heads, kD, kBN) ||
             !TmapEncoder::token_tensor(&mVq, Vq, (uint64_t)nQ, n_heads, kD, kBN)) return PAFU_ERR_CUDA;
     } else { mKq = mQ; mVq = mQ; }
     Params p;
-    p.st = st; p.n_heads = n_heads; p.has_chunk = Kq != nullptr; p.scale = scale;
-    p.O = O; p.LSE = LSE; p.status = status; p.total_Lq = nQ;
+    p.st = st; p.n_heads = n_heads; p.has_chunk = has_chunk; p.scale = scale;
+    p.O = O; p.LSE = LSE; p.status = status; p.pieces = pieces; p.total_Lq = nQ; p.total_cost = cost;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return PAFU_ERR_CUDA;
         attr_set = true;
     }
-    attn_tc_kernel<<<(unsigned)items, kThreads, kSmemBytes, stream>>>(mQ, mKc, mVc, mKq, mVq, p);
-    return cuda_ok(cudaGetLastError());
+    const int grid = grid_for(cost);
+    attn_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(mQ, mKc, mVc, mKq, mVq, p);
+    if (cudaGetLastError() != cudaSuccess) return PAFU_ERR_CUDA;
+    if (grid > 1) {
+        attn_tc_merge_kernel<<<grid, 256, 0, stream>>>(p, grid);
+        if (cudaGetLastError() != cudaSuccess) return PAFU_ERR_CUDA;
+    }
+    return PAFU_OK;
 }
 
 }  // namespace attn_tc
