@@ -6,8 +6,9 @@
 // Work decomposition.  An "item" is 256 query rows of one head of one stream, handled as two
 // 128-row "slots" that share every K/V tile (each tile is fetched once per 256 rows).  The
 // grid is persistent: one CTA per SM.  All items' key tiles are laid end to end and cut into
-// equal contiguous shares, one per CTA (cost of a tile = number of live slots), so every SM
-// gets the same amount of tensor work whatever the item count.  A CTA whose share covers only
+// equal contiguous shares, one per CTA (a tile with both slots live costs 4 units, with one
+// slot 3: a lone slot has no partner to hide its softmax behind), so every SM gets the same
+// amount of work whatever the item count.  A CTA whose share covers only
 // part of an item's keys writes an unnormalised partial (O, running max, row sum) to the
 // workspace; a second small kernel merges the partials of each split item in key order, which
 // keeps the result deterministic.
@@ -83,6 +84,8 @@ struct Seg {
                          // earlier CTA; 1: begins an item that a later CTA continues
 };
 
+constexpr int kCost2 = 4, kCost1 = 3;   // cost of one key tile with two / one live slots
+
 struct StreamCost {
     int64_t nqp, nt, head_cost;
     int tail_slots;
@@ -95,7 +98,7 @@ __host__ __device__ inline StreamCost stream_cost(const StreamTable& st, int s, 
     c.nqp = (lq + 2 * kBM - 1) / (2 * kBM);
     c.tail_slots = (lq - (c.nqp - 1) * 2 * kBM > kBM) ? 2 : 1;
     c.nt = (nB + kBN - 1) / kBN + (has_chunk ? (lq + kBN - 1) / kBN : 0);
-    c.head_cost = (lq > 0) ? c.nt * (2 * (c.nqp - 1) + c.tail_slots) : 0;
+    c.head_cost = (lq > 0) ? c.nt * (kCost2 * (c.nqp - 1) + (c.tail_slots == 2 ? kCost2 : kCost1)) : 0;
     return c;
 }
 
@@ -127,20 +130,21 @@ struct SegIter {
             g.stream = s;
             g.head = (int)(c / sc.head_cost);
             const int64_t r = c % sc.head_cost;
-            const int64_t full = sc.nt * 2 * (sc.nqp - 1);
+            const int64_t full = sc.nt * kCost2 * (sc.nqp - 1);
             int64_t qp, rr;
-            if (r < full) { qp = r / (2 * sc.nt); rr = r % (2 * sc.nt); g.n_slots = 2; }
+            if (r < full) { qp = r / (kCost2 * sc.nt); rr = r % (kCost2 * sc.nt); g.n_slots = 2; }
             else { qp = sc.nqp - 1; rr = r - full; g.n_slots = sc.tail_slots; }
+            const int unit = g.n_slots == 2 ? kCost2 : kCost1;
             g.q0 = qp * 2 * kBM;
             g.Lq = p.st.cu_Lq[s + 1] - p.st.cu_Lq[s];
             g.nB = p.st.cu_B[s + 1] - p.st.cu_B[s];
             g.nC = p.has_chunk ? g.Lq : 0;
             g.nt1 = (int)((g.nB + kBN - 1) / kBN);
             g.nt = (int)sc.nt;
-            const int64_t item_start = cur - rr, item_end = item_start + sc.nt * g.n_slots;
-            g.t0 = (int)(rr / g.n_slots);
+            const int64_t item_start = cur - rr, item_end = item_start + sc.nt * unit;
+            g.t0 = (int)(rr / unit);
             if (c1 >= item_end) { g.t1 = g.nt; cur = item_end; }
-            else { g.t1 = (int)((c1 - item_start) / g.n_slots); cur = c1; }
+            else { g.t1 = (int)((c1 - item_start) / unit); cur = c1; }
             if (g.t1 > g.t0) {
                 g.piece = (g.t0 == 0 && g.t1 == g.nt) ? -1 : (g.t0 > 0 ? 0 : 1);
                 return true;
@@ -154,6 +158,30 @@ __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// packed fp32 pairs (two lanes per instruction on the FMA pipe)
+__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
@@ -214,13 +242,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
             if (p.has_chunk) { prefetch_tmap(&mKq); prefetch_tmap(&mVq); }
             SegIter iter(p, blockIdx.x, gridDim.x);
             Seg g;
-            uint32_t ring = 0, qcnt[2] = {0, 0};
+            uint32_t ring = 0, qcnt0 = 0, qcnt1 = 0;      // scalars: a runtime-indexed array would live in local memory
             bool ok = true;
             while (ok && iter.next(p, g)) {
                 const int qrow = (int)(p.st.cu_Lq[g.stream] + g.q0);
                 for (int s = 0; s < g.n_slots && ok; ++s) {
-                    if (abort_flag || !mbar_wait(q_empty(s), (qcnt[s] & 1u) ^ 1u)) { fail(100); ok = false; break; }
-                    ++qcnt[s];
+                    const uint32_t qc = s ? qcnt1 : qcnt0;
+                    if (abort_flag || !mbar_wait(q_empty(s), (qc & 1u) ^ 1u)) { fail(100); ok = false; break; }
+                    if (s) ++qcnt1; else ++qcnt0;
                     mbar_arrive_expect_tx(q_full(s), kTileBytes);
                     tma_load_3d(sQ + s * kTileBytes, &mQ, q_full(s), 0, g.head, qrow + s * kBM);
                     tma_load_3d(sQ + s * kTileBytes + kHalfBytes, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
@@ -276,9 +305,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
             };
             SegIter iter(p, blockIdx.x, gridDim.x);
             Seg g;
-            uint32_t ring = 0, qcnt[2] = {0, 0}, pcnt[2] = {0, 0};
+            uint32_t ring = 0, qcnt0 = 0, qcnt1 = 0, pcnt0 = 0, pcnt1 = 0;
             while (ok && iter.next(p, g)) {
-                for (int s = 0; s < g.n_slots; ++s) { wait(q_full(s), qcnt[s] & 1u, 201); ++qcnt[s]; }
+                for (int s = 0; s < g.n_slots; ++s) {
+                    wait(q_full(s), (s ? qcnt1 : qcnt0) & 1u, 201);
+                    if (s) ++qcnt1; else ++qcnt0;
+                }
                 {   // S(t0) for every live slot
                     const int st = ring % kStages;
                     wait(kv_full(st), (ring / kStages) & 1u, 202);
@@ -295,9 +327,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                     wait(kv_full(stv), (rv / kStages) & 1u, 203);
                     if (more) wait(kv_full(stk), (rk / kStages) & 1u, 204);
                     for (int s = 0; s < g.n_slots && ok; ++s) {
-                        wait(p_full(s), pcnt[s] & 1u, 205);
+                        wait(p_full(s), (s ? pcnt1 : pcnt0) & 1u, 205);
                         if (!ok) break;
-                        ++pcnt[s];
+                        if (s) ++pcnt1; else ++pcnt0;
                         tc_fence_after_sync();
                         issue_pv(s, stv, j == g.t0);
                         if (more) { issue_qk(s, stk); umma_commit(s_full(s)); }
@@ -350,9 +382,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                     for (int c = 0; c < 128; ++c)
                         if (c >= left) sr[c] = 0xff800000u;   // -inf
                 }
-                float mx = __uint_as_float(sr[0]);
+                // row maximum: four independent chains of 3-input max
+                float mx4[4];
 #pragma unroll
-                for (int c = 1; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sr[c]));
+                for (int q = 0; q < 4; ++q) {
+                    float m = fmaxf(__uint_as_float(sr[32 * q]), __uint_as_float(sr[32 * q + 1]));
+#pragma unroll
+                    for (int c = 2; c < 32; c += 2)
+                        m = fmax3(m, __uint_as_float(sr[32 * q + c]), __uint_as_float(sr[32 * q + c + 1]));
+                    mx4[q] = m;
+                }
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 if (j == g.t0) {
                     m_used = mx;
                 } else if (__any_sync(0xffffffffu, (mx - m_used) * sl2 > kRescaleThresholdLog2)) {
@@ -372,20 +412,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                         PAFU_TMEM_ST_X32(tO + c * 32, orr);
                     }
                 }
-                const float mb = m_used * sl2;
-                float rs = 0.f;
+                // p = 2^(s * sl2 - m * sl2): packed FMA for the exponent, packed adds for the sum
+                const float mb = -m_used * sl2;
+                const uint64_t sl2_2 = pack2(__float_as_uint(sl2), __float_as_uint(sl2));
+                const uint64_t mb_2 = pack2(__float_as_uint(mb), __float_as_uint(mb));
+                uint64_t rs2[2] = {0ull, 0ull};
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     uint32_t pk[32];
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[64 * h + 2 * c]), sl2, -mb));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[64 * h + 2 * c + 1]), sl2, -mb));
-                        rs += p0 + p1;
+                        float e0, e1;
+                        unpack2(ffma2(pack2(sr[64 * h + 2 * c], sr[64 * h + 2 * c + 1]), sl2_2, mb_2), e0, e1);
+                        const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
+                        rs2[c & 1] = fadd2(rs2[c & 1], pack2(__float_as_uint(p0), __float_as_uint(p1)));
                         pk[c] = pack_bf16(p0, p1);
                     }
                     PAFU_TMEM_ST_X32(tS + 32 * h, pk);
                 }
+                float r0, r1, r2, r3;
+                unpack2(rs2[0], r0, r1);
+                unpack2(rs2[1], r2, r3);
+                const float rs = (r0 + r1) + (r2 + r3);
                 l_sum += rs;
                 tmem_wait_st();
                 tc_fence_before_sync();
