@@ -281,21 +281,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
         if (elect_one()) {
             const uint32_t idesc_qk = make_idesc_bf16(kBM, kBN, false, false);
             const uint32_t idesc_pv = make_idesc_bf16(kBM, kD, false, true);
+            // Descriptors differ from tile to tile only in the 14-bit start-address field, so the
+            // constant part is built once and the address (in 16-byte units) is added per MMA.
+            const uint64_t desc_k = make_smem_desc_sw128(0, 16, 1024);             // K-major Q / K
+            const uint64_t desc_v = make_smem_desc_sw128(0, kHalfBytes, 1024);     // MN-major V
             auto issue_qk = [&](int slot, int stage) {
-                const uint32_t a = sQ + slot * kTileBytes, b = sKV + stage * kTileBytes;
+                const uint64_t a = desc_k + ((sQ + slot * kTileBytes) >> 4);
+                const uint64_t b = desc_k + ((sKV + stage * kTileBytes) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-                    umma_ss(tmem + slot * kBN, make_smem_desc_sw128(a + off, 16, 1024),
-                            make_smem_desc_sw128(b + off, 16, 1024), idesc_qk, kk > 0);
+                    const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+                    umma_ss(tmem + slot * kBN, a + off, b + off, idesc_qk, kk > 0);
                 }
             };
             auto issue_pv = [&](int slot, int stage, bool first) {
-                const uint32_t b = sKV + stage * kTileBytes;
+                const uint64_t b = desc_v + ((sKV + stage * kTileBytes) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < kBN / 16; ++kk)
-                    umma_ts(tmem + 256 + slot * kD, tmem + slot * kBN + kk * 8,
-                            make_smem_desc_sw128(b + kk * 2048, kHalfBytes, 1024), idesc_pv,
+                    umma_ts(tmem + 256 + slot * kD, tmem + slot * kBN + kk * 8, b + kk * (2048 >> 4), idesc_pv,
                             !(first && kk == 0));
             };
             bool ok = true;
@@ -327,7 +330,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                     wait(kv_full(stv), (rv / kStages) & 1u, 203);
                     if (more) wait(kv_full(stk), (rk / kStages) & 1u, 204);
                     for (int s = 0; s < g.n_slots && ok; ++s) {
-                        wait(p_full(s), (s ? pcnt1 : pcnt0) & 1u, 205);
+                        if (ok && (abort_flag || !mbar_wait_spin(p_full(s), (s ? pcnt1 : pcnt0) & 1u))) { fail(205); ok = false; }
                         if (!ok) break;
                         if (s) ++pcnt1; else ++pcnt0;
                         tc_fence_after_sync();
@@ -363,25 +366,68 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
             float m_used = -INFINITY, l_sum = 0.f;
             for (int j = g.t0; j < g.t1; ++j) {
                 {
-                    const bool w = mbar_wait(s_full(slot), scnt & 1u) && !abort_flag;
+                    const bool w = mbar_wait_spin(s_full(slot), scnt & 1u) && !abort_flag;
                     if (!__all_sync(0xffffffffu, w)) { fail(301); ok = false; break; }   // warp-uniform
                     ++scnt;
                 }
                 tc_fence_after_sync();
                 uint32_t sr[128];
-                PAFU_TMEM_LD_X32(tS, sr);
-                PAFU_TMEM_LD_X32(tS + 32, sr + 32);
-                PAFU_TMEM_LD_X32(tS + 64, sr + 64);
-                PAFU_TMEM_LD_X32(tS + 96, sr + 96);
-                tmem_wait_ld();
-                // ragged end of a key segment
                 const bool seg2 = j >= g.nt1;
                 const int64_t left = (seg2 ? g.nC - (int64_t)(j - g.nt1) * kBN : g.nB - (int64_t)j * kBN);
-                if (left < kBN) {
+                const float sl2n = sl2;
+                const uint64_t sl2_2 = pack2(__float_as_uint(sl2n), __float_as_uint(sl2n));
+                // Fast path (every tile but a run's first and a segment's ragged last): the
+                // exponentials use the running maximum as it stands, so they start as soon as
+                // the first quarter of S has arrived and overlap the remaining TMEM loads; the
+                // tile's own maximum is only needed for the (rare) rescale decision at the end.
+                bool full_pass = (j == g.t0) || (left < kBN);
+                if (!full_pass) {
+                    const float mbf = -m_used * sl2;
+                    const uint64_t mb_2 = pack2(__float_as_uint(mbf), __float_as_uint(mbf));
+                    uint64_t rs2[2] = {0ull, 0ull};
+                    float mx4[4];
+                    PAFU_TMEM_LD_X32(tS, sr);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 128; ++c)
-                        if (c >= left) sr[c] = 0xff800000u;   // -inf
+                    for (int c = 0; c < 4; ++c) {
+                        if (c < 3) PAFU_TMEM_LD_X32(tS + 32 * (c + 1), sr + 32 * (c + 1));
+                        uint32_t pk[16];
+                        float m = -INFINITY;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const uint32_t u0 = sr[32 * c + 2 * i], u1 = sr[32 * c + 2 * i + 1];
+                            float e0, e1;
+                            unpack2(ffma2(pack2(u0, u1), sl2_2, mb_2), e0, e1);
+                            const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
+                            rs2[i & 1] = fadd2(rs2[i & 1], pack2(__float_as_uint(p0), __float_as_uint(p1)));
+                            pk[i] = pack_bf16(p0, p1);
+                            m = fmax3(m, __uint_as_float(u0), __uint_as_float(u1));
+                        }
+                        mx4[c] = m;
+                        PAFU_TMEM_ST_X16(tS + 16 * c, pk);
+                        if (c < 3) tmem_wait_ld();
+                    }
+                    const float mxf = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                    full_pass = __any_sync(0xffffffffu, (mxf - m_used) * sl2 > kRescaleThresholdLog2);
+                    if (!full_pass) {
+                        float r0, r1, r2, r3;
+                        unpack2(rs2[0], r0, r1);
+                        unpack2(rs2[1], r2, r3);
+                        l_sum += (r0 + r1) + (r2 + r3);
+                    }
+                } else {
+                    PAFU_TMEM_LD_X32(tS, sr);
+                    PAFU_TMEM_LD_X32(tS + 32, sr + 32);
+                    PAFU_TMEM_LD_X32(tS + 64, sr + 64);
+                    PAFU_TMEM_LD_X32(tS + 96, sr + 96);
+                    tmem_wait_ld();
+                    if (left < kBN) {          // ragged end of a key segment
+#pragma unroll
+                        for (int c = 0; c < 128; ++c)
+                            if (c >= left) sr[c] = 0xff800000u;   // -inf
+                    }
                 }
+                if (full_pass) {
                 // row maximum: four independent chains of 3-input max
                 float mx4[4];
 #pragma unroll
@@ -414,7 +460,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 }
                 // p = 2^(s * sl2 - m * sl2): packed FMA for the exponent, packed adds for the sum
                 const float mb = -m_used * sl2;
-                const uint64_t sl2_2 = pack2(__float_as_uint(sl2), __float_as_uint(sl2));
                 const uint64_t mb_2 = pack2(__float_as_uint(mb), __float_as_uint(mb));
                 uint64_t rs2[2] = {0ull, 0ull};
 #pragma unroll
@@ -435,6 +480,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 unpack2(rs2[1], r2, r3);
                 const float rs = (r0 + r1) + (r2 + r3);
                 l_sum += rs;
+                }   // full_pass
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(p_full(slot));

@@ -51,6 +51,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     return done != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, P;\n\t}\n"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
 // Every wait is bounded: after kWaitLimitNs without completion the caller gets `false`,
 // records the failure and unwinds; nothing in these kernels can spin forever.
 constexpr uint64_t kWaitLimitNs = 400ull * 1000 * 1000;   // 0.4 s
@@ -64,6 +73,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
         if (global_timer_ns() - t0 > kWaitLimitNs) return false;
     }
+}
+
+// Low-latency variant for waits on the critical path: polls without suspending first (a
+// suspended try_wait can wake late), then falls back to the bounded wait above.
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity) {
+#pragma unroll 1
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
+    return mbar_wait(bar, parity);
 }
 
 // ------------------------------------------------------------------------------- fences
