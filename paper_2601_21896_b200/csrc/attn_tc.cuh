@@ -56,7 +56,7 @@ constexpr float kRescaleThresholdLog2 = 8.0f;
 constexpr int kRegsLaunch = 168, kRegsLow = 80, kRegsHigh = 208;
 static_assert((kRegsLaunch - kRegsLow) * 128 >= (kRegsHigh - kRegsLaunch) * 256,
               "setmaxnreg.inc would wait forever");
-constexpr int kMaxGrid = 256;
+constexpr int kMaxGrid = kMaxPersistentGrid;
 // one partial: O [256][128] fp32, then m [256], then l [256]
 constexpr int kPieceFloats = 2 * kBM * kD + 2 * 2 * kBM;
 constexpr size_t kPieceBytes = (size_t)kPieceFloats * 4;
@@ -602,18 +602,7 @@ attn_tc_merge_kernel(const __grid_constant__ Params p, int n_cta) {
     }
 }
 
-inline int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-            n = v < kMaxGrid ? v : kMaxGrid;
-        else
-            return 148;      // no device visible (sizing queries on a build host)
-    }
-    return n;
-}
+inline int sm_count() { return device_sm_count(); }
 
 inline int grid_for(int64_t cost) {
     const int sms = sm_count();

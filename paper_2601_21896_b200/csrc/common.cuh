@@ -26,6 +26,22 @@ constexpr int kStatusWordTimeout = 0;   // non-zero: a bounded wait ran out
 inline pafu_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? PAFU_OK : PAFU_ERR_CUDA; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// SM count of the current device (148 when no device is visible, e.g. sizing queries on a
+// build host); capped so per-CTA tables stay small.
+constexpr int kMaxPersistentGrid = 256;
+inline int device_sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v < kMaxPersistentGrid ? v : kMaxPersistentGrid;
+        else
+            return 148;
+    }
+    return n;
+}
+
 // Launchers (each enqueues on `stream` and returns the launch status).
 pafu_status launch_score(const pafu_head& head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
                          float* scores, void* ws, size_t ws_bytes, cudaStream_t stream);

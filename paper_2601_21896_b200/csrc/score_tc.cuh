@@ -1,0 +1,259 @@
+// Salience Estimation Head on the tensor cores (Sec. 3.3; Appendix A "S-MLP"):
+//   s_t = mean_o( W2 act(W1 x_t + b1) + b2 ),  optionally sigmoid(s_t).
+//
+// The first layer is a [tokens x d_in] x [d_in x d_hidden] contraction with ~d_hidden flop
+// per input byte, i.e. on the tensor-core ridge; it runs as a tcgen05 GEMM and everything
+// after it is fused into the accumulator read-out, so HBM traffic is "read X once, write
+// 4 bytes per token".  Since the mean over outputs is linear, the second layer folds to
+//   w2m[h] = mean_o W2[o, h],  b2m = mean_o b2[o],  s = sum_h w2m[h] act(a_h + b1[h]) + b2m.
+//
+// Persistent CTAs, one per SM, each taking 128-token tiles round-robin.  Warp roles:
+//   warps 0-7  read-out: thread = token row (TMEM lane); warps w and w+4 split the hidden
+//              columns of the same 32 rows; bias, activation, dot with w2m, row reduction
+//   warp  8    MMA issuer (A = X tile, B = W1 tile, both K-major in shared memory)
+//   warp  9    TMA loader, 4-stage ring of {X 128x64, W1 256x64} tiles
+// Hidden units are processed in chunks of up to 256 (one accumulator of 256 TMEM columns);
+// two accumulators alternate so the read-out of one chunk overlaps the MMAs of the next.
+// All mbarrier waits are bounded (see sm100.cuh).
+#pragma once
+#include "common.cuh"
+#include "sm100.cuh"
+
+namespace pafu {
+namespace score_tc {
+
+using namespace sm100;
+
+constexpr int kBM = 128;             // tokens per tile
+constexpr int kBK = 64;              // reduction slice per stage (one 128-byte swizzle row)
+constexpr int kNMax = 256;           // hidden units per accumulator
+constexpr int kStages = 4;
+constexpr int kThreads = 384;
+constexpr int kXBytes = kBM * kBK * 2;          // 16 KiB
+constexpr int kWBytes = kNMax * kBK * 2;        // 32 KiB
+constexpr int kStageBytes = kXBytes + kWBytes;
+constexpr int kMaxHidden = 1024;
+constexpr int kSmemBytes = kStages * kStageBytes + 2 * kMaxHidden * 4 + 2 * kBM * 4 + 256 + 1024;
+
+struct Params {
+    int64_t n_tokens;
+    int d_in, d_hidden, d_out, act, final;
+    const uint16_t* w2;
+    const uint16_t* b1;
+    const uint16_t* b2;
+    float* scores;
+    int* status;
+};
+
+__device__ __forceinline__ float bf16_bits(uint16_t b) { return __uint_as_float(((uint32_t)b) << 16); }
+
+__device__ __forceinline__ float ex2f(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float rcpf(float x) { float y; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+
+// GELU in its exact form x * Phi(x) = x/2 * (1 + erf(x / sqrt 2)), erf by the rational
+// approximation of Abramowitz & Stegun 7.1.26 (absolute error below 1.5e-7).
+__device__ __forceinline__ float gelu_erf(float x) {
+    const float z = fabsf(x) * 0.70710678118654752f;
+    const float t = rcpf(fmaf(0.3275911f, z, 1.0f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    const float e = ex2f(-z * z * 1.4426950408889634f);
+    const float erf_abs = fmaf(-poly * t, e, 1.0f);
+    const float erf_v = copysignf(erf_abs, x);
+    return 0.5f * x * (1.0f + erf_v);
+}
+__device__ __forceinline__ float silu(float x) { return x * rcpf(1.0f + ex2f(-x * 1.4426950408889634f)); }
+
+template <int ACT>
+__device__ __forceinline__ float act_fn(float x) { return ACT == PAFU_ACT_GELU ? gelu_erf(x) : silu(x); }
+
+template <int ACT>
+__global__ void __launch_bounds__(kThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ CUtensorMap mW,
+                const __grid_constant__ Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sStage = smem_u32(smem);
+    float* w2m = reinterpret_cast<float*>(smem + kStages * kStageBytes);
+    float* b1s = w2m + kMaxHidden;
+    float* half_sum = b1s + kMaxHidden;                      // [2][kBM]: partial of column-half 1
+    uint64_t* bars = reinterpret_cast<uint64_t*>(half_sum + 2 * kBM);
+    const uint32_t bar0 = smem_u32(bars);
+    auto full = [&](int st) { return bar0 + 8 * st; };
+    auto empty = [&](int st) { return bar0 + 8 * (kStages + st); };
+    auto acc_full = [&](int b) { return bar0 + 8 * (2 * kStages + b); };
+    auto acc_empty = [&](int b) { return bar0 + 8 * (2 * kStages + 2 + b); };
+    const uint32_t halves_bar = bar0 + 8 * (2 * kStages + 4);   // column-half 1 -> column-half 0
+    __shared__ uint32_t tmem_base_sh;
+    __shared__ volatile int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t n_tiles = (p.n_tokens + kBM - 1) / kBM;
+    const int n_chunks = (p.d_hidden + kNMax - 1) / kNMax;
+    const int n_k = p.d_in / kBK;
+
+    if (tid == 0) {
+        for (int st = 0; st < kStages; ++st) { mbar_init(full(st), 1); mbar_init(empty(st), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 8); }
+        mbar_init(halves_bar, 4);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 8) { tmem_alloc(smem_u32(&tmem_base_sh), 512); tmem_relinquish(); }
+    // folded second layer and first-layer bias, fp32 in shared memory
+    for (int h = tid; h < p.d_hidden; h += kThreads) {
+        float m = 0.f;
+        for (int o = 0; o < p.d_out; ++o) m += bf16_bits(p.w2[(int64_t)o * p.d_hidden + h]);
+        w2m[h] = m / (float)p.d_out;
+        b1s[h] = p.b1 ? bf16_bits(p.b1[h]) : 0.f;
+    }
+    float b2m = 0.f;
+    if (p.b2) {
+        for (int o = 0; o < p.d_out; ++o) b2m += bf16_bits(p.b2[o]);
+        b2m /= (float)p.d_out;
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_base_sh;
+
+    auto fail = [&](int code) {
+        abort_flag = 1;
+        atomicCAS(p.status, 0, code);
+    };
+
+    if (warp == 9) {
+        // ---------------------------------------------------------------------- TMA loader
+        if (elect_one()) {
+            prefetch_tmap(&mX); prefetch_tmap(&mW);
+            uint32_t ring = 0;
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                for (int ch = 0; ch < n_chunks && ok; ++ch) {
+                    for (int k = 0; k < n_k; ++k, ++ring) {
+                        const int st = ring % kStages;
+                        if (abort_flag || !mbar_wait(empty(st), ((ring / kStages) & 1u) ^ 1u)) { fail(401); ok = false; break; }
+                        const uint32_t dst = sStage + st * kStageBytes;
+                        mbar_arrive_expect_tx(full(st), kStageBytes);
+                        tma_load_2d(dst, &mX, full(st), k * kBK, (int)(tile * kBM));
+                        tma_load_2d(dst + kXBytes, &mW, full(st), k * kBK, ch * kNMax);
+                    }
+                }
+            }
+            if (!ok)
+                for (uint32_t r = ring > (uint32_t)kStages ? ring - kStages : 0; r < ring; ++r)
+                    mbar_wait(full(r % kStages), (r / kStages) & 1u);
+        }
+        __syncwarp();
+    } else if (warp == 8) {
+        // ---------------------------------------------------------------------- MMA issuer
+        if (elect_one()) {
+            const uint64_t desc0 = make_smem_desc_sw128(0, 16, 1024);
+            uint32_t ring = 0, acc_it = 0;
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                for (int ch = 0; ch < n_chunks && ok; ++ch, ++acc_it) {
+                    const int buf = acc_it & 1;
+                    const int nc = min(kNMax, p.d_hidden - ch * kNMax);
+                    const uint32_t idesc = make_idesc_bf16(kBM, nc, false, false);
+                    if (abort_flag || !mbar_wait(acc_empty(buf), ((acc_it >> 1) & 1u) ^ 1u)) { fail(402); ok = false; break; }
+                    tc_fence_after_sync();
+                    for (int k = 0; k < n_k; ++k, ++ring) {
+                        const int st = ring % kStages;
+                        if (abort_flag || !mbar_wait(full(st), (ring / kStages) & 1u)) { fail(403); ok = false; break; }
+                        tc_fence_after_sync();
+                        const uint64_t a = desc0 + ((sStage + st * kStageBytes) >> 4);
+                        const uint64_t b = desc0 + ((sStage + st * kStageBytes + kXBytes) >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < kBK / 16; ++kk)
+                            umma_ss(tmem + buf * kNMax, a + kk * 2, b + kk * 2, idesc, (k | kk) != 0);
+                        umma_commit(empty(st));
+                    }
+                    if (ok) umma_commit(acc_full(buf));
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp < 8) {
+        // ------------------------------------------------------------------------ read-out
+        const int quad = warp & 3, half = warp >> 2;
+        const uint32_t lane_base = ((uint32_t)(quad * 32)) << 16;
+        const int row = quad * 32 + lane;
+        uint32_t acc_it = 0, tile_it = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
+            float part = 0.f;
+            for (int ch = 0; ch < n_chunks; ++ch, ++acc_it) {
+                const int buf = acc_it & 1;
+                const int nc = min(kNMax, p.d_hidden - ch * kNMax);
+                {
+                    const bool w = mbar_wait(acc_full(buf), (acc_it >> 1) & 1u) && !abort_flag;
+                    if (!__all_sync(0xffffffffu, w)) { fail(404); ok = false; break; }
+                }
+                tc_fence_after_sync();
+                // 16-column groups of this chunk alternate between the two warps of a row
+                for (int g16 = half; g16 < nc / 16; g16 += 2) {
+                    uint32_t r[16];
+                    PAFU_TMEM_LD_X16(tmem + buf * kNMax + lane_base + g16 * 16, r);
+                    tmem_wait_ld();
+                    const int h0 = ch * kNMax + g16 * 16;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        part = fmaf(w2m[h0 + i], act_fn<ACT>(__uint_as_float(r[i]) + b1s[h0 + i]), part);
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty(buf));
+            }
+            if (!ok) break;
+            // combine the two column halves of each row
+            float* hs = half_sum + (tile_it & 1) * kBM;
+            if (half == 1) {
+                hs[row] = part;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(halves_bar);
+            } else {
+                const bool w = mbar_wait(halves_bar, tile_it & 1u) && !abort_flag;
+                if (!__all_sync(0xffffffffu, w)) { fail(405); ok = false; break; }
+                const int64_t t = tile * kBM + row;
+                if (t < p.n_tokens) {
+                    float v = part + hs[row] + b2m;
+                    if (p.final == PAFU_FINAL_SIGMOID) v = rcpf(1.0f + ex2f(-v * 1.4426950408889634f));
+                    p.scores[t] = v;
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 8) tmem_dealloc(tmem, 512);
+}
+
+inline pafu_status launch(const pafu_head& head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
+                          float* scores, int* status, int sm_count, cudaStream_t stream) {
+    CUtensorMap mX, mW;
+    if (!TmapEncoder::matrix(&mX, X, (uint64_t)n_tokens, (uint64_t)head.d_in, (uint64_t)ldx, kBM)) return PAFU_ERR_CUDA;
+    if (!TmapEncoder::matrix(&mW, head.w1, (uint64_t)head.d_hidden, (uint64_t)head.d_in, (uint64_t)head.d_in, kNMax))
+        return PAFU_ERR_CUDA;
+    Params p;
+    p.n_tokens = n_tokens; p.d_in = head.d_in; p.d_hidden = head.d_hidden; p.d_out = head.d_out;
+    p.act = head.act; p.final = head.final; p.w2 = head.w2; p.b1 = head.b1; p.b2 = head.b2;
+    p.scores = scores; p.status = status;
+    const int64_t n_tiles = (n_tokens + kBM - 1) / kBM;
+    const int grid = (int)(n_tiles < sm_count ? n_tiles : sm_count);
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(score_tc_kernel<PAFU_ACT_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(score_tc_kernel<PAFU_ACT_SILU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+            return PAFU_ERR_CUDA;
+        attr_set = true;
+    }
+    if (head.act == PAFU_ACT_GELU) score_tc_kernel<PAFU_ACT_GELU><<<grid, kThreads, kSmemBytes, stream>>>(mX, mW, p);
+    else score_tc_kernel<PAFU_ACT_SILU><<<grid, kThreads, kSmemBytes, stream>>>(mX, mW, p);
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace score_tc
+}  // namespace pafu
