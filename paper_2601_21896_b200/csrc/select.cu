@@ -2,8 +2,8 @@
 // Sec. 4.1): kept = [0, n_sink) U top-k salient of the middle U [T - n_recent, T), written as
 // ascending token indices, ties to the lower index.
 //
-// The step moves a few hundred KB, so it is latency-bound: one launch, one CTA of 1024
-// threads per stream, scores read from L2.
+// The step moves a few hundred KB, so it is latency-bound: one CTA of 1024 threads per
+// stream, scores read from L2 (once, into registers, when the stream is small enough).
 //   1. fp32 scores map to order-preserving 32-bit keys (-0 folded onto +0, NaN lowest).
 //   2. MSB-first radix select (4 passes of 8 bits, shared-memory histograms) finds the key of
 //      the k-th largest candidate and how many candidates equal to it are still needed.
@@ -51,8 +51,187 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
     return warp_sums[warp] + inc - v;
 }
 
+constexpr int kSelRows = 32;                          // candidates per thread held in registers
+constexpr int kSelRegCap = kSelRows * kSelThreads;    // 32768 candidates
+constexpr int kSelList = 2048;                        // survivors of the first pass kept in shared memory
+
+// Streams with at most kSelRegCap candidates: every candidate key is loaded once (all loads in
+// flight together) and stays in registers for the three radix passes (12 + 10 + 10 bits) and
+// the emission.  Candidate j of the stream sits in row j / 1024 of thread j % 1024, so a warp
+// ballot per row plus one block scan over the 32 x 32 (row, warp) counts gives every kept
+// candidate its ascending output slot.
 __global__ void __launch_bounds__(kSelThreads)
-select_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __restrict__ idx) {
+select_regs_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __restrict__ idx) {
+    __shared__ int hist[4096];
+    __shared__ int cnt[kSelRows * 32];
+    __shared__ uint32_t list[kSelList];
+    __shared__ int warp_sums[33];
+    __shared__ uint32_t sh_prefix;
+    __shared__ int sh_krem, sh_bin, sh_nlist;
+
+    const int s = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t T64 = st.cu_T[s + 1] - st.cu_T[s];
+    const int64_t B64 = st.cu_B[s + 1] - st.cu_B[s];
+    if (B64 >= T64) return;                               // the streaming kernel writes the identity
+    const int T = (int)T64;
+    const int ns = (int)st.n_sink[s], nr = (int)st.n_recent[s];
+    const int k = (int)st.k[s];
+    const int c0 = ns, M = T - nr - ns;
+    if (M > kSelRegCap) return;                           // the streaming kernel owns this stream
+    const float* sc = scores + st.cu_T[s] + c0;
+    int32_t* out = idx + st.cu_B[s];
+
+    uint32_t key[kSelRows];
+#pragma unroll
+    for (int i = 0; i < kSelRows; ++i) {
+        const int j = i * kSelThreads + tid;
+        key[i] = (j < M) ? score_key(__ldg(sc + j)) : 0u;
+    }
+    // sink and recent tokens are kept as they are
+    for (int t = tid; t < ns; t += kSelThreads) out[t] = t;
+    for (int t = tid; t < nr; t += kSelThreads) out[ns + k + t] = T - nr + t;
+
+    uint32_t thr = 0xffffffffu;
+    int need_eq = 0, eq_total = 0;
+    if (k > 0) {
+        uint32_t prefix = 0u, mask = 0u;
+        int k_rem = k;
+        int shift = 32;
+        int n_list = -1;                                  // >= 0: survivors are in list[]
+#pragma unroll 1
+        for (int pass = 0; pass < 3; ++pass) {
+            const int bits = pass == 0 ? 12 : 10;
+            const int nb = 1 << bits;
+            shift -= bits;
+            for (int b = tid; b < nb; b += kSelThreads) hist[b] = 0;
+            __syncthreads();
+            if (n_list >= 0) {
+                // few candidates share the leading digit(s): work on the compacted list
+                for (int j = tid; j < n_list; j += kSelThreads) {
+                    const uint32_t kv = list[j];
+                    if ((kv & mask) == prefix) atomicAdd(&hist[(kv >> shift) & (uint32_t)(nb - 1)], 1);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < kSelRows; ++i) {
+                    const bool in = (i * kSelThreads + tid < M) && ((key[i] & mask) == prefix);
+                    const uint32_t digit = (key[i] >> shift) & (uint32_t)(nb - 1);
+                    // a warp whose live lanes all hold one digit (equal or saturated scores) adds once
+                    const unsigned act = __ballot_sync(0xffffffffu, in);
+                    if (act != 0u) {
+                        const uint32_t d0 = __shfl_sync(0xffffffffu, digit, __ffs(act) - 1);
+                        const bool uniform = __all_sync(0xffffffffu, !in || digit == d0);
+                        if (uniform) { if (lane == __ffs(act) - 1) atomicAdd(&hist[d0], __popc(act)); }
+                        else if (in) atomicAdd(&hist[digit], 1);
+                    }
+                }
+            }
+            __syncthreads();
+            // thread t owns bins nb-1 - t*bpt ... downwards; the exclusive scan of the per-thread
+            // counts is the number of matching candidates in all higher bins
+            const int bpt = nb >= kSelThreads ? nb / kSelThreads : 1;
+            int mine = 0;
+            if (tid * bpt < nb)
+                for (int i = 0; i < bpt; ++i) mine += hist[nb - 1 - (tid * bpt + i)];
+            int total;
+            int above = block_exclusive_scan(mine, warp_sums, &total);
+            if (tid * bpt < nb) {
+                for (int i = 0; i < bpt; ++i) {
+                    const int b = nb - 1 - (tid * bpt + i);
+                    const int c = hist[b];
+                    if (above < k_rem && k_rem <= above + c) {
+                        sh_prefix = prefix | ((uint32_t)b << shift);
+                        sh_krem = k_rem - above;
+                        sh_bin = c;
+                    }
+                    above += c;
+                }
+            }
+            if (tid == 0) sh_nlist = 0;
+            __syncthreads();
+            prefix = sh_prefix;
+            k_rem = sh_krem;
+            mask |= (uint32_t)(nb - 1) << shift;
+            eq_total = sh_bin;                            // after the last pass: keys equal to thr
+            if (pass == 0 && sh_bin <= kSelList) {
+                // gather the candidates that share the winning leading digit
+#pragma unroll
+                for (int i = 0; i < kSelRows; ++i)
+                    if ((i * kSelThreads + tid < M) && ((key[i] & mask) == prefix))
+                        list[atomicAdd(&sh_nlist, 1)] = key[i];
+                __syncthreads();
+                n_list = sh_nlist;
+            }
+        }
+        thr = prefix;
+        need_eq = k_rem;
+    }
+
+    // ---- ordered emission.  First the ties: rank of every candidate equal to the threshold.
+    const unsigned lt_mask = (1u << lane) - 1u;
+    uint32_t keep_bits = 0u;
+    int total;
+    if (need_eq == eq_total) {
+        // every candidate equal to the threshold is taken: no tie to break
+#pragma unroll
+        for (int i = 0; i < kSelRows; ++i)
+            if ((i * kSelThreads + tid < M) && k > 0 && key[i] >= thr) keep_bits |= 1u << i;
+    } else {
+        uint32_t eq_bits = 0u;                            // bit i: row i equals the threshold
+#pragma unroll
+        for (int i = 0; i < kSelRows; ++i) {
+            const bool eq = (i * kSelThreads + tid < M) && key[i] == thr;
+            const unsigned b = __ballot_sync(0xffffffffu, eq);
+            if (lane == 0) cnt[i * 32 + warp] = __popc(b);
+            if (eq) eq_bits |= 1u << i;
+        }
+        __syncthreads();
+        {
+            const int v = cnt[tid];
+            const int ex = block_exclusive_scan(v, warp_sums, &total);
+            __syncthreads();
+            cnt[tid] = ex;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kSelRows; ++i) {
+            const bool valid = i * kSelThreads + tid < M;
+            const bool eq = (eq_bits >> i) & 1u;
+            const unsigned b = __ballot_sync(0xffffffffu, eq);
+            const int rank = cnt[i * 32 + warp] + __popc(b & lt_mask);
+            const bool keep = valid && (key[i] > thr || (eq && rank < need_eq));
+            if (keep) keep_bits |= 1u << i;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kSelRows; ++i) {
+        const unsigned b = __ballot_sync(0xffffffffu, (keep_bits >> i) & 1u);
+        if (lane == 0) cnt[i * 32 + warp] = __popc(b);
+    }
+    __syncthreads();
+    {
+        const int v = cnt[tid];
+        const int ex = block_exclusive_scan(v, warp_sums, &total);
+        __syncthreads();
+        cnt[tid] = ex;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kSelRows; ++i) {
+        const bool keep = (keep_bits >> i) & 1u;
+        const unsigned b = __ballot_sync(0xffffffffu, keep);
+        if (keep) out[ns + cnt[i * 32 + warp] + __popc(b & lt_mask)] = c0 + i * kSelThreads + tid;
+    }
+}
+
+// Streams with more candidates than the register kernel holds: keys are re-read from L2 in
+// every pass (4 passes of 8 bits), and each thread emits a contiguous token range.
+__global__ void __launch_bounds__(kSelThreads)
+select_stream_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __restrict__ idx) {
+    if (st.cu_T[blockIdx.x + 1] - st.cu_T[blockIdx.x] - st.n_sink[blockIdx.x] - st.n_recent[blockIdx.x] <= kSelRegCap &&
+        st.cu_B[blockIdx.x + 1] - st.cu_B[blockIdx.x] < st.cu_T[blockIdx.x + 1] - st.cu_T[blockIdx.x]) return;   // the register kernel owns this stream
     __shared__ int hist[256];
     __shared__ int warp_sums[33];
     __shared__ uint32_t sh_prefix;
@@ -152,7 +331,16 @@ select_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __restr
 pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* idx,
                           cudaStream_t stream) {
     if (st.n_streams == 0 || st.cu_B[st.n_streams] == 0) return PAFU_OK;
-    select_kernel<<<st.n_streams, kSelThreads, 0, stream>>>(scores, st, idx);
+    // both kernels run over all streams; each stream is handled by exactly one of them
+    bool any_regs = false, any_stream = false;
+    for (int s = 0; s < st.n_streams; ++s) {
+        const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
+        const bool regs = B < T && T - st.n_sink[s] - st.n_recent[s] <= kSelRegCap;
+        any_regs |= regs;
+        any_stream |= !regs;
+    }
+    if (any_regs) select_regs_kernel<<<st.n_streams, kSelThreads, 0, stream>>>(scores, st, idx);
+    if (any_stream) select_stream_kernel<<<st.n_streams, kSelThreads, 0, stream>>>(scores, st, idx);
     return cuda_ok(cudaGetLastError());
 }
 
