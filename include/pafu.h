@@ -50,7 +50,8 @@ enum {
     PAFU_ERR_WORKSPACE_TOO_SMALL = 4,
     PAFU_ERR_MISALIGNED = 5,         /* a device pointer is not 16-byte aligned */
     PAFU_ERR_CUDA = 6,               /* a CUDA runtime/driver call failed (launch error, no device) */
-    PAFU_ERR_TIMEOUT = 7             /* a bounded device-side wait ran out (pafu_workspace_status) */
+    PAFU_ERR_TIMEOUT = 7,            /* a bounded device-side wait ran out (pafu_workspace_status) */
+    PAFU_ERR_TOO_LARGE = 8           /* problem exceeds the built-in scratch of pafu_chunk_attn_noalloc */
 };
 
 /* Activation between the two linear layers of the salience head. */
@@ -175,6 +176,33 @@ pafu_status pafu_chunk_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_
                             const int64_t* cu_B, const uint16_t* Kq, const uint16_t* Vq,
                             const pafu_shape* shape, float scale, uint16_t* O, float* LSE,
                             void* ws, size_t ws_bytes, void* stream);
+
+/* Chunk attention without a workspace - the paper has no counterpart; this entry point exists
+ * for callers that are not allowed to allocate device memory: code running inside another
+ * framework's memory plan or a fixed-memory service, plug-ins handed only their input and
+ * output buffers, and anything else that must not call cudaMalloc (directly or through an
+ * allocating library) on its hot path.  It computes exactly what pafu_chunk_attn computes
+ * (same arguments, same layouts, d_head = 128 only, every stream needs at least one key), but
+ * the scratch the kernel needs lives in a device array built into the library:
+ * PAFU_NOALLOC_SCRATCH_BYTES bytes that every GPU which loads the library holds until the
+ * process exits.  The call allocates and frees nothing.
+ *   - Limit: sum over streams of query rows, times n_heads, must not exceed
+ *     PAFU_NOALLOC_MAX_QUERY_HEAD_ROWS; larger problems return PAFU_ERR_TOO_LARGE and nothing
+ *     is launched.  The built-in scratch holds the partial results of 31 thread blocks, so the
+ *     kernel runs on at most 31 SMs: expect it to be several times slower than pafu_chunk_attn.
+ *   - The first call on each device looks up the device address of the built-in array (a
+ *     runtime query, no allocation).  Make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps whatever the last call left there; the call
+ *     clears the part that must start at zero itself.  Two calls that overlap on the GPU (on
+ *     different streams, or from different host threads) race on it: serialise them.
+ *   - A bounded wait that runs out cannot be reported (there is no workspace to read back);
+ *     use pafu_chunk_attn where that matters. */
+#define PAFU_NOALLOC_SCRATCH_BYTES (8u * 1024u * 1024u)
+#define PAFU_NOALLOC_MAX_QUERY_HEAD_ROWS 65536
+pafu_status pafu_chunk_attn_noalloc(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
+                                    const int64_t* cu_B, const uint16_t* Kq, const uint16_t* Vq,
+                                    const pafu_shape* shape, float scale, uint16_t* O, float* LSE,
+                                    void* stream);
 
 /* Arguments of one whole layer step (Algorithm 2's order: score, Top-k, Select, attend). */
 typedef struct pafu_step_args {

@@ -23,11 +23,12 @@ FINAL_NONE, FINAL_SIGMOID = 0, 1
 
 STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET",
                 3: "PAFU_ERR_UNSUPPORTED_SHAPE", 4: "PAFU_ERR_WORKSPACE_TOO_SMALL",
-                5: "PAFU_ERR_MISALIGNED", 6: "PAFU_ERR_CUDA", 7: "PAFU_ERR_TIMEOUT"}
+                5: "PAFU_ERR_MISALIGNED", 6: "PAFU_ERR_CUDA", 7: "PAFU_ERR_TIMEOUT",
+                8: "PAFU_ERR_TOO_LARGE"}
 
 EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
            "pafu_workspace_status", "pafu_score", "pafu_select", "pafu_compact",
-           "pafu_chunk_attn", "pafu_step", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host"]
+           "pafu_chunk_attn", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host"]
 
 
 class PafuError(RuntimeError):
@@ -103,6 +104,9 @@ def lib() -> ctypes.CDLL:
         L.pafu_chunk_attn.restype = i32
         L.pafu_chunk_attn.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.POINTER(CShape),
                                       ctypes.c_float, vp, vp, vp, sz, vp]
+        L.pafu_chunk_attn_noalloc.restype = i32
+        L.pafu_chunk_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.POINTER(CShape),
+                                              ctypes.c_float, vp, vp, vp]
         L.pafu_step.restype = i32
         L.pafu_step.argtypes = [ctypes.POINTER(CStepArgs), vp]
         L.pafu_step_timed.restype = i32
@@ -223,6 +227,15 @@ def pafu_chunk_attn(Q, Kc, Vc, cu_B, Kq, Vq, shape: Shape, scale: float, O, LSE=
                                  ctypes.byref(shape.c), float(scale), _ptr(O), _ptr(LSE), _ptr(ws),
                                  0 if ws is None else ws.numel() * ws.element_size(), _stream()),
            "pafu_chunk_attn")
+
+
+def pafu_chunk_attn_noalloc(Q, Kc, Vc, cu_B, Kq, Vq, shape: Shape, scale: float, O, LSE=None) -> None:
+    """Chunk attention that takes no workspace: its scratch is a fixed array inside the library
+    (see include/pafu.h for the size limit and the rule that calls must not overlap)."""
+    cu_B = np.ascontiguousarray(cu_B, dtype=np.int64)
+    _check(lib().pafu_chunk_attn_noalloc(_ptr(Q), _ptr(Kc), _ptr(Vc), _ptr(cu_B), _ptr(Kq), _ptr(Vq),
+                                         ctypes.byref(shape.c), float(scale), _ptr(O), _ptr(LSE),
+                                         _stream()), "pafu_chunk_attn_noalloc")
 
 
 def step_args(shape: Shape, head: Head, policy, K, V, Q, Kq, Vq, scale, scores, idx, Kc, Vc, SLc,

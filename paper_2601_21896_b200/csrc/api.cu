@@ -89,6 +89,7 @@ const char* pafu_status_string(pafu_status s) {
         case PAFU_ERR_MISALIGNED: return "device pointer not 16-byte aligned";
         case PAFU_ERR_CUDA: return "CUDA call failed";
         case PAFU_ERR_TIMEOUT: return "bounded device wait ran out";
+        case PAFU_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }

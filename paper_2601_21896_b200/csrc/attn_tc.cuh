@@ -627,7 +627,7 @@ inline size_t workspace_bytes() { return (size_t)sm_count() * 2 * kPieceBytes; }
 inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
                           const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
                           int32_t n_heads, float scale, uint16_t* O, float* LSE, int* status,
-                          float* pieces, cudaStream_t stream) {
+                          float* pieces, cudaStream_t stream, int max_ctas = 0) {
     const int n = st.n_streams;
     const int64_t nQ = st.cu_Lq[n], nB = st.cu_B[n];
     const int has_chunk = Kq != nullptr;
@@ -652,7 +652,8 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
             return PAFU_ERR_CUDA;
         attr_set = true;
     }
-    const int grid = grid_for(cost);
+    int grid = grid_for(cost);
+    if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;   // caller's scratch holds fewer partials
     attn_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(mQ, mKc, mVc, mKq, mVq, p);
     if (cudaGetLastError() != cudaSuccess) return PAFU_ERR_CUDA;
     if (grid > 1) {
