@@ -542,21 +542,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
-// Merges the partials of every item that was split across CTAs.  Block b owns the item that
-// CTA b of the main kernel began (its last run, stored as piece 1) and adds the following
-// CTAs' continuation pieces (their first run, piece 0) in key order.
+// Merges the partials of every item that was split across CTAs.  Blocks 2b and 2b+1 own the
+// two slots of the item that CTA b of the main kernel began (its last run, stored as piece 1)
+// and add the following CTAs' continuation pieces (their first run, piece 0) in key order.
+// Each warp handles four rows at a time so that all their loads are in flight together.
+constexpr int kMergeRows = 4;
 __global__ void __launch_bounds__(256)
 attn_tc_merge_kernel(const __grid_constant__ Params p, int n_cta) {
     __shared__ int piece_cta[kMaxGrid];
     __shared__ int n_pieces_sh;
-    const int b = blockIdx.x;
+    const int b = blockIdx.x >> 1, slot = blockIdx.x & 1;
     Seg g, last;
     bool have = false;
     {
         SegIter iter(p, b, n_cta);
         while (iter.next(p, g)) { last = g; have = true; }
     }
-    if (!have || last.piece != 1) return;      // block-uniform
+    if (!have || last.piece != 1 || slot >= last.n_slots) return;      // block-uniform
     if (threadIdx.x == 0) {
         int n = 0, t = last.t1;
         piece_cta[n++] = b;
@@ -571,34 +573,50 @@ attn_tc_merge_kernel(const __grid_constant__ Params p, int n_cta) {
     __syncthreads();
     const int n_pieces = n_pieces_sh;
     const float sl2 = p.scale * 1.4426950408889634f;
-    const int lane = threadIdx.x & 31, sub = threadIdx.x >> 5;   // 8 rows per pass, 32 float4 per row
-    const int n_rows = last.n_slots * kBM;
-    for (int r = sub; r < n_rows; r += 8) {
-        const int64_t row = last.q0 + r;
-        if (row >= last.Lq) break;
-        float M = -INFINITY;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;   // 32 float4 per row
+    const float* __restrict__ pieces = p.pieces;
+    for (int r0 = warp * kMergeRows; r0 < kBM; r0 += 8 * kMergeRows) {
+        float M[kMergeRows], L[kMergeRows];
+        float4 acc[kMergeRows];
+#pragma unroll
+        for (int q = 0; q < kMergeRows; ++q) { M[q] = -INFINITY; L[q] = 0.f; acc[q] = make_float4(0.f, 0.f, 0.f, 0.f); }
         for (int i = 0; i < n_pieces; ++i) {
-            const float* piece = p.pieces + ((size_t)piece_cta[i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
-            M = fmaxf(M, piece[2 * kBM * kD + r]);
+            const float* piece = pieces + ((size_t)piece_cta[i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
+#pragma unroll
+            for (int q = 0; q < kMergeRows; ++q) M[q] = fmaxf(M[q], piece[2 * kBM * kD + slot * kBM + r0 + q]);
         }
-        float L = 0.f;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int i = 0; i < n_pieces; ++i) {
-            const float* piece = p.pieces + ((size_t)piece_cta[i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
-            const float w = fast_exp2((piece[2 * kBM * kD + r] - M) * sl2);
-            L += w * piece[2 * kBM * kD + 2 * kBM + r];
-            const float4 v = reinterpret_cast<const float4*>(piece + (size_t)r * kD)[lane];
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+            const float* piece = pieces + ((size_t)piece_cta[i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
+            float w[kMergeRows], l[kMergeRows];
+            float4 v[kMergeRows];
+#pragma unroll
+            for (int q = 0; q < kMergeRows; ++q) {
+                const int r = slot * kBM + r0 + q;
+                w[q] = piece[2 * kBM * kD + r];
+                l[q] = piece[2 * kBM * kD + 2 * kBM + r];
+                v[q] = reinterpret_cast<const float4*>(piece + (size_t)r * kD)[lane];
+            }
+#pragma unroll
+            for (int q = 0; q < kMergeRows; ++q) {
+                const float ww = fast_exp2((w[q] - M[q]) * sl2);
+                L[q] += ww * l[q];
+                acc[q].x += ww * v[q].x; acc[q].y += ww * v[q].y; acc[q].z += ww * v[q].z; acc[q].w += ww * v[q].w;
+            }
         }
-        const float inv = (L > 0.f) ? 1.0f / L : 0.f;
-        uint16_t* dst = p.O + ((p.st.cu_Lq[last.stream] + row) * p.n_heads + last.head) * kD + lane * 4;
-        uint2 o;
-        o.x = pack_bf16(acc.x * inv, acc.y * inv);
-        o.y = pack_bf16(acc.z * inv, acc.w * inv);
-        *reinterpret_cast<uint2*>(dst) = o;
-        if (p.LSE != nullptr && lane == 0)
-            p.LSE[(int64_t)last.head * p.total_Lq + p.st.cu_Lq[last.stream] + row] =
-                (L > 0.f) ? M * p.scale + logf(L) : -INFINITY;
+#pragma unroll
+        for (int q = 0; q < kMergeRows; ++q) {
+            const int64_t row = last.q0 + slot * kBM + r0 + q;
+            if (row >= last.Lq) continue;
+            const float inv = (L[q] > 0.f) ? 1.0f / L[q] : 0.f;
+            uint16_t* dst = p.O + ((p.st.cu_Lq[last.stream] + row) * p.n_heads + last.head) * kD + lane * 4;
+            uint2 o;
+            o.x = pack_bf16(acc[q].x * inv, acc[q].y * inv);
+            o.y = pack_bf16(acc[q].z * inv, acc[q].w * inv);
+            *reinterpret_cast<uint2*>(dst) = o;
+            if (p.LSE != nullptr && lane == 0)
+                p.LSE[(int64_t)last.head * p.total_Lq + p.st.cu_Lq[last.stream] + row] =
+                    (L[q] > 0.f) ? M[q] * p.scale + logf(L[q]) : -INFINITY;
+        }
     }
 }
 
@@ -657,7 +675,7 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
     attn_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(mQ, mKc, mVc, mKq, mVq, p);
     if (cudaGetLastError() != cudaSuccess) return PAFU_ERR_CUDA;
     if (grid > 1) {
-        attn_tc_merge_kernel<<<grid, 256, 0, stream>>>(p, grid);
+        attn_tc_merge_kernel<<<2 * grid, 256, 0, stream>>>(p, grid);
         if (cudaGetLastError() != cudaSuccess) return PAFU_ERR_CUDA;
     }
     return PAFU_OK;
