@@ -96,6 +96,37 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def recorded_traffic(w):
+    """DRAM bytes per attention launch from the committed ncu summary, or None when the
+    summary is for another workload or the kernel source changed since the counters were taken."""
+    import hashlib
+    import re
+    path = os.path.join(ROOT, "profiles", "attn_tc_kernel_%s.md" % w.name)
+    src = os.path.join(ROOT, "paper_2601_21896_b200", "csrc", "attn_tc.cuh")
+    if not (os.path.exists(path) and os.path.exists(src)):
+        return None
+    text = open(path).read()
+    m_b = re.search(r"traffic_bytes_per_launch:\s*(\d+)", text)
+    m_h = re.search(r"source_sha256:\s*([0-9a-f]{64})", text)
+    if not (m_b and m_h):
+        return None
+    if hashlib.sha256(open(src, "rb").read()).hexdigest() != m_h.group(1):
+        return None
+    return int(m_b.group(1))
+
+
+def launches_per_step(w):
+    """Kernels of this library one step launches: score, select (register and/or streaming
+    variant), compact, attention (+ the merge of split items for d_head 128)."""
+    regs = stream = False
+    for t, b in zip(w.T, w.budget):
+        if b < t and t - min(w.n_sink, b) - min(w.n_recent, b) <= 32768:
+            regs = True
+        else:
+            stream = True
+    return 1 + int(regs) + int(stream) + 1 + (2 if w.d_head == 128 else 1)
+
+
 def pick_workload(name: str):
     from paper_2601_21896_b200 import workloads as wl
     if name in ("wan1.3b_layer", "default"):
@@ -157,7 +188,7 @@ def oracle_sampled_step(w, d, n_score_tokens, n_rows, seed=0):
 
 def cpu_baseline(w, d, budget_s=15.0):
     import oracle
-    probe = oracle_sampled_step(w, d, 64, 1 * w.n_streams)
+    probe = oracle_sampled_step(w, d, 256, 8 * w.n_streams)
     per_tok = probe["score_s"] / probe["score_tokens"]
     per_row = probe["attn_s"] / probe["attn_rows"]
     n_tok = int(max(64, min(sum(w.T), 0.3 * budget_s / max(per_tok, 1e-9))))
@@ -182,7 +213,7 @@ def run_reference(args):
     steps = args.steps if args.steps is not None else 3
     warmup = args.warmup if args.warmup is not None else 1
     d = wl.make_layer(w)
-    probe = oracle_sampled_step(w, d, 64, w.n_streams)
+    probe = oracle_sampled_step(w, d, 256, 8 * w.n_streams)
     per_step_budget = max(0.2, 90.0 / (steps + warmup))
     n_tok = int(max(16, min(sum(w.T), 0.3 * per_step_budget / (probe["score_s"] / probe["score_tokens"]))))
     n_rows = int(max(w.n_streams, min(sum(w.Lq), 0.6 * per_step_budget / (probe["attn_s"] / probe["attn_rows"]))))
@@ -214,6 +245,7 @@ def run_ours(args):
     import paper_2601_21896_b200 as pafu
     from paper_2601_21896_b200 import workloads as wl
     from paper_2601_21896_b200.harness import Layer
+    from paper_2601_21896_b200 import sharding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -232,8 +264,9 @@ def run_ours(args):
     # independent layer units per rank (weak scaling: no data-path collective)
     n_sets = args.sets
     layers, host0 = [], None
-    for i in range(n_sets):
-        d = wl.make_layer(w, seed=0, layer=rank * n_sets + i)
+    my_units = sharding.units_for_rank(world * n_sets, rank, world)
+    for i, unit in enumerate(my_units):
+        d = wl.make_layer(w, seed=0, layer=unit)
         if i == 0:
             host0 = d
         layers.append(Layer(w, d, want_lse=False, want_slc=True))
@@ -273,11 +306,7 @@ def run_ours(args):
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     for L in layers:
         L.check_status()
-    total_ms = start.elapsed_time(end)
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = sharding.max_over_ranks(start.elapsed_time(end), device="cuda")
     parts = np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(4)] for ev in step_events])
     k_ms = parts.mean(axis=0)          # score, select, compact, attn
     ms_per_step = total_ms / steps
@@ -307,11 +336,7 @@ def run_ours(args):
         pafu.pafu_step_host(hargs, arena)
     e1.record(stream)
     torch.cuda.synchronize()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = sharding.max_over_ranks(e0.elapsed_time(e1) / e2e_steps, device="cuda")
     h2d = sum(int(v.numel() * v.element_size()) for v in hin.values())
     d2h = int(h_scores.numel() * 4 + h_idx.numel() * 4 + h_O.numel() * 2)
     e2e_value = world * work["attn_flops"] / (e2e_ms * 1e-3) / 1e12
@@ -335,7 +360,7 @@ def run_ours(args):
                    "l2": "inputs larger than L2: %d independent layer buffer sets (>= 300 MB each) used "
                          "round-robin, no flush" % n_sets},
         "roofline": {"kernel": "chunk attention", "bound": "tensor", "achieved": attn_tf, "peak": peak_tf,
-                     "unit": "TFLOP/s", "frac": attn_tf / peak_tf, "traffic": None,
+                     "unit": "TFLOP/s", "frac": attn_tf / peak_tf, "traffic": recorded_traffic(w),
                      "peak_source": "%s, %s" % (peaks["source"], "burst" if burst else "sustained")},
         "kernels": {
             "score": {"ms": k_ms[0], "GB/s": gbs(work["score_bytes"], k_ms[0]),
@@ -356,7 +381,7 @@ def run_ours(args):
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "api": "pafu_step_host (pinned host buffers)"},
-        "gpu_launches": 4 * steps,
+        "gpu_launches": launches_per_step(w) * steps,
     }
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, host0, budget_s=args.cpu_seconds)
