@@ -214,7 +214,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
             mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1); mbar_init(s_full(s), 1);
-            mbar_init(p_full(s), kBM); mbar_init(o_done(s), 1);
+            mbar_init(p_full(s), 4); mbar_init(o_done(s), 1);   // p_full: one arrival per softmax warp
         }
         for (int st = 0; st < kStages; ++st) { mbar_init(kv_full(st), 1); mbar_init(kv_empty(st), 1); }
         abort_flag = 0;
@@ -483,7 +483,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 }   // full_pass
                 tmem_wait_st();
                 tc_fence_before_sync();
-                mbar_arrive(p_full(slot));
+                __syncwarp();
+                if ((tid & 31) == 0) mbar_arrive(p_full(slot));
             }
             if (!ok) break;
             {
