@@ -6,8 +6,8 @@
 // Work decomposition.  An "item" is 256 query rows of one head of one stream, handled as two
 // 128-row "slots" that share every K/V tile (each tile is fetched once per 256 rows).  The
 // grid is persistent: one CTA per SM.  All items' key tiles are laid end to end and cut into
-// equal contiguous shares, one per CTA (a tile with both slots live costs 4 units, with one
-// slot 3: a lone slot has no partner to hide its softmax behind), so every SM gets the same
+// equal contiguous shares, one per CTA (a tile with both slots live costs 8 units, with one
+// slot 7: a lone slot has no partner to hide its softmax behind), so every SM gets the same
 // amount of work whatever the item count.  A CTA whose share covers only
 // part of an item's keys writes an unnormalised partial (O, running max, row sum) to the
 // workspace; a second small kernel merges the partials of each split item in key order, which
@@ -84,7 +84,7 @@ struct Seg {
                          // earlier CTA; 1: begins an item that a later CTA continues
 };
 
-constexpr int kCost2 = 4, kCost1 = 3;   // cost of one key tile with two / one live slots
+constexpr int kCost2 = 8, kCost1 = 7;   // cost of one key tile with two / one live slots (measured ratio)
 
 struct StreamCost {
     int64_t nqp, nt, head_cost;
@@ -546,9 +546,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
 // Merges the partials of every item that was split across CTAs.  Blocks 2b and 2b+1 own the
 // two slots of the item that CTA b of the main kernel began (its last run, stored as piece 1)
 // and add the following CTAs' continuation pieces (their first run, piece 0) in key order.
-// Each warp handles four rows at a time so that all their loads are in flight together.
+// Each of the 32 warps handles four rows, so all loads of a block are in flight together.
 constexpr int kMergeRows = 4;
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 attn_tc_merge_kernel(const __grid_constant__ Params p, int n_cta) {
     __shared__ int piece_cta[kMaxGrid];
     __shared__ int n_pieces_sh;
@@ -576,7 +576,7 @@ attn_tc_merge_kernel(const __grid_constant__ Params p, int n_cta) {
     const float sl2 = p.scale * 1.4426950408889634f;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;   // 32 float4 per row
     const float* __restrict__ pieces = p.pieces;
-    for (int r0 = warp * kMergeRows; r0 < kBM; r0 += 8 * kMergeRows) {
+    for (int r0 = warp * kMergeRows; r0 < kBM; r0 += 32 * kMergeRows) {   // one pass with 32 warps
         float M[kMergeRows], L[kMergeRows];
         float4 acc[kMergeRows];
 #pragma unroll
@@ -676,7 +676,7 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
     attn_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(mQ, mKc, mVc, mKq, mVq, p);
     if (cudaGetLastError() != cudaSuccess) return PAFU_ERR_CUDA;
     if (grid > 1) {
-        attn_tc_merge_kernel<<<2 * grid, 256, 0, stream>>>(p, grid);
+        attn_tc_merge_kernel<<<2 * grid, 1024, 0, stream>>>(p, grid);
         if (cudaGetLastError() != cudaSuccess) return PAFU_ERR_CUDA;
     }
     return PAFU_OK;
