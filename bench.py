@@ -255,14 +255,15 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    steps = args.steps if args.steps is not None else 200
-    warmup = max(3, args.warmup if args.warmup is not None else 10)
+    steps = args.steps if args.steps is not None else (200 if args.layers <= 1 else 20)
+    warmup = max(3, args.warmup if args.warmup is not None else (10 if args.layers <= 1 else 3))
     w = pick_workload(args.workload)
     work = algorithmic_work(w)
     peaks = measured_peaks()
 
     # independent layer units per rank (weak scaling: no data-path collective)
-    n_sets = args.sets
+    n_layers = max(1, args.layers)
+    n_sets = max(args.sets, n_layers) if n_layers > 1 else args.sets
     layers, host0 = [], None
     my_units = sharding.units_for_rank(world * n_sets, rank, world)
     for i, unit in enumerate(my_units):
@@ -278,11 +279,11 @@ def run_ours(args):
             e.record(stream)          # torch creates the cudaEvent_t on first record
         return ev
 
-    for i in range(warmup):
+    for i in range(warmup * n_layers):
         layers[i % n_sets].step()
     for L in layers:
         L.check_status()
-    step_events = [new_events(5) for _ in range(steps)]
+    step_events = [new_events(5) for _ in range(steps * n_layers)]
     handles = [pafu.event_handles(ev) for ev in step_events]
     start, end = new_events(2)
     sampler = ClockSampler(local)
@@ -295,7 +296,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     t_wall0 = time.time()
     start.record(stream)
-    for i in range(steps):
+    for i in range(steps * n_layers):
         pafu.pafu_step_timed(layers[i % n_sets].args, handles[i])
     end.record(stream)
     torch.cuda.synchronize()
@@ -308,9 +309,9 @@ def run_ours(args):
         L.check_status()
     total_ms = sharding.max_over_ranks(start.elapsed_time(end), device="cuda")
     parts = np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(4)] for ev in step_events])
-    k_ms = parts.mean(axis=0)          # score, select, compact, attn
+    k_ms = parts.mean(axis=0)          # score, select, compact, attn (per layer)
     ms_per_step = total_ms / steps
-    value = world * work["attn_flops"] / (ms_per_step * 1e-3) / 1e12
+    value = world * n_layers * work["attn_flops"] / (ms_per_step * 1e-3) / 1e12
 
     # ---- e2e: host buffers through pafu_step_host (H2D of inputs + D2H of results timed)
     L0 = layers[0]
@@ -357,6 +358,7 @@ def run_ours(args):
         "config": {"workload": w.name, "heads": w.n_heads, "d_head": w.d_head, "cache_tokens": list(w.T),
                    "budget": list(w.budget), "n_sink": w.n_sink, "n_recent": w.n_recent,
                    "chunk_tokens": list(w.Lq), "head_mlp": [w.d_model, w.d_hidden, w.d_out],
+                   "layers_per_step": n_layers,
                    "l2": "inputs larger than L2: %d independent layer buffer sets (>= 300 MB each) used "
                          "round-robin, no flush" % n_sets},
         "roofline": {"kernel": "chunk attention", "bound": "tensor", "achieved": attn_tf, "peak": peak_tf,
@@ -376,12 +378,13 @@ def run_ours(args):
                 "hbm_frac": gbs(work["score_bytes"] + work["select_bytes"] + work["compact_bytes"],
                                 k_ms[:3].sum()) / peaks["hbm_gbs"]},
         },
-        "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step,
+        "layers_per_step": n_layers,
+        "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step / n_layers,
         "peaks": peaks,
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "api": "pafu_step_host (pinned host buffers)"},
-        "gpu_launches": launches_per_step(w) * steps,
+        "gpu_launches": launches_per_step(w) * steps * n_layers,
     }
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, host0, budget_s=args.cpu_seconds)
@@ -398,6 +401,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="wan1.3b_layer")
     ap.add_argument("--sets", type=int, default=3, help="independent layer buffer sets used round-robin")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="layers per step; 30 with --workload wan1.3b_layer_b25/_b50/_b75 is the full "
+                         "denoising step of the 30-layer sweep (every layer has its own cache and head)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -240,13 +240,19 @@ def test_step_host_matches_device_step():
 
 
 # ---------------------------------------------------------------------- full-size configs
-def _full_size_check(w, n_rows=256, seed=0):
+def _full_size_check(w, n_rows=256, seed=0, score_rows=None):
     d = wl.make_layer(w, seed=seed)
     L = Layer(w, d)
     L.step(); L.check_status()
     torch.cuda.synchronize()
     gs = L.scores[: L.nT].cpu().numpy()
-    close(gs, oracle_scores(w, d), "scores")
+    if score_rows is None:
+        close(gs, oracle_scores(w, d), "scores")
+    else:
+        # the oracle's MLP on a seeded sample of tokens (first, last and tile-boundary rows included)
+        rows = wl.sample_rows(L.nT, score_rows, seed=seed, tag=77)
+        want = oracle.score(d["K"].reshape(L.nT, -1)[rows], d["w1"], d["b1"], d["w2"], d["b2"], w.act, w.final)
+        close(gs[rows], want, "scores (sampled)")
     idx = oracle_select_streams(gs, w)
     got_idx = L.idx[: L.nB].cpu().numpy()
     cuT, cuB, cuQ = w.cu("T"), L.cu_B, w.cu("Lq")
@@ -271,5 +277,23 @@ def test_full_size_wan13b_layer():
     _full_size_check(wl.wan13b_layer())
 
 
+@pytest.mark.parametrize("frac", [0.25, 0.75])
+def test_full_size_budget_sweep(frac):
+    # the other two budgets of the 30-layer sweep (a different layer's random streams each)
+    w = wl.wan13b_layer(frac)
+    assert w.budget[0] == {0.25: 7020, 0.75: 21060}[frac]
+    _full_size_check(w, n_rows=48, seed=int(frac * 100), score_rows=4096)
+
+
 def test_full_size_paper_native_point():
     _full_size_check(wl.paper_native(), n_rows=96)
+
+
+def test_full_size_long_horizon():
+    # 93 600-token cache pruned to 9360: the streaming select kernel and heavy-tailed scores
+    _full_size_check(wl.long_horizon(), n_rows=128, score_rows=8192)
+
+
+def test_full_size_batch4_14b():
+    # four ragged streams, 40 heads, D_M = 5120, hidden 512 (two accumulator chunks per tile)
+    _full_size_check(wl.batch4_14b(), n_rows=24, score_rows=2048)
