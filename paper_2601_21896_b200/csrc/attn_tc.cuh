@@ -16,19 +16,22 @@
 // Warp roles inside a CTA (384 threads):
 //   warps 0-3  softmax of slot 0 (thread = query row = TMEM lane)
 //   warps 4-7  softmax of slot 1
-//   warp  8    MMA issuer: S = Q K^T (both operands in shared memory) and O += P V
-//              (P read from tensor memory, V from shared memory, MN-major)
-//   warp  9    TMA loader: Q tiles per item, K/V tiles through a 5-stage ring that runs
-//              ahead across item boundaries
-//   warps 10-11 idle (they complete the third warpgroup so registers can be re-balanced)
-// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; the bf16 P tile
-// overwrites the first 64 columns of its S tile.  While one slot runs its softmax the tensor
-// core works on the other slot's two products.
+//   warps 8,10 MMA issuers, one per slot: S = Q K^T (both operands in shared memory) and
+//              O += P V (P read from tensor memory, V from shared memory, MN-major).  One thread
+//              can start a tcgen05.mma only about every 100 clocks while the tensor core
+//              finishes a 128x128x16 one in 64, hence an issuing thread per slot
+//   warp  9    TMA loader: Q tiles per item, 64-key K/V tiles through a 10-stage ring that
+//              runs ahead across item boundaries
+//   warp  11   idle (completes the third warpgroup so registers can be re-balanced)
+// Tensor memory (512 columns): per slot two S buffers of 64 fp32 columns and one O accumulator
+// of 128; the bf16 P tile overwrites the first 32 columns of its S buffer.  S is double
+// buffered so that S(j+1) = Q K_{j+1}^T is already finished when the softmax of tile j ends:
+// the softmax warps never wait for the tensor core in steady state, and the issuer's order
+// "P(j) ready -> O += P(j) V_j -> S(j+2)" keeps the buffer reuse safe without extra barriers.
 //
 // Online softmax with lazy rescaling: the running maximum only moves when the new tile
 // exceeds it by more than 2^8 in the exponent, so the O accumulator is rarely rescaled; when
-// it is, the slot's own softmax warps do it between "S ready" (which implies the previous
-// P V product has finished) and "P ready" (which releases the next one).
+// it is, the slot's own softmax warps do it after waiting for the previous P V product.
 //
 // Every mbarrier wait is bounded.  A wait that runs out sets the status word, raises a CTA-wide
 // abort flag, and all roles fall through to the common exit where TMEM is released.
@@ -43,12 +46,14 @@ using namespace sm100;
 
 constexpr int kD = 128;
 constexpr int kBM = 128;            // query rows per slot
-constexpr int kBN = 128;            // keys per tile
-constexpr int kStages = 5;          // K/V ring depth (each stage one 128 x 128 bf16 tile)
-constexpr int kThreads = 384;       // 3 warpgroups: softmax 0, softmax 1, {MMA, loader, 2 idle}
-constexpr int kTileBytes = kBN * kD * 2;      // 32 KiB
-constexpr int kHalfBytes = kTileBytes / 2;    // one [128 rows x 64 cols] swizzled half
-constexpr int kSmemBytes = 2 * kTileBytes + kStages * kTileBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int kBN = 64;             // keys per tile
+constexpr int kStages = 10;         // K/V ring depth (each stage one 64 x 128 bf16 tile)
+constexpr int kThreads = 384;       // 3 warpgroups: softmax 0, softmax 1, {2 MMA issuers, loader, 1 idle}
+constexpr int kQBytes = kBM * kD * 2;         // 32 KiB: one slot's Q tile
+constexpr int kQHalf = kQBytes / 2;           // one [128 rows x 64 cols] swizzled half
+constexpr int kTileBytes = kBN * kD * 2;      // 16 KiB: one K or V tile
+constexpr int kHalfBytes = kTileBytes / 2;    // one [64 rows x 64 cols] swizzled half
+constexpr int kSmemBytes = 2 * kQBytes + kStages * kTileBytes + 1024 /*align*/ + 512 /*barriers*/;
 constexpr float kRescaleThresholdLog2 = 8.0f;
 // Register re-balancing.  With 384 threads the kernel launches with 168 registers per thread.
 // setmaxnreg.inc blocks until the registers exist, so what the third warpgroup gives up must
@@ -196,16 +201,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sQ = smem_u32(smem);                       // 2 slots x 32 KiB
-    const uint32_t sKV = sQ + 2 * kTileBytes;                 // ring
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kTileBytes + kStages * kTileBytes);
+    const uint32_t sKV = sQ + 2 * kQBytes;                    // ring
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kQBytes + kStages * kTileBytes);
     const uint32_t bar0 = smem_u32(bars);
     auto q_full = [&](int s) { return bar0 + 8 * (0 + s); };
     auto q_empty = [&](int s) { return bar0 + 8 * (2 + s); };
-    auto s_full = [&](int s) { return bar0 + 8 * (4 + s); };
-    auto p_full = [&](int s) { return bar0 + 8 * (6 + s); };
-    auto o_done = [&](int s) { return bar0 + 8 * (8 + s); };
-    auto kv_full = [&](int st) { return bar0 + 8 * (10 + st); };
-    auto kv_empty = [&](int st) { return bar0 + 8 * (10 + kStages + st); };
+    auto s_full = [&](int s, int b) { return bar0 + 8 * (4 + 2 * s + b); };
+    // P-ready is per S buffer as well: the softmax may finish tile j+1 (whose S was computed
+    // early) before the issuer has looked at tile j, and a single barrier would be lapped
+    auto p_full = [&](int s, int b) { return bar0 + 8 * (8 + 2 * s + b); };
+    auto pv_done = [&](int s) { return bar0 + 8 * (12 + s); };
+    auto o_done = [&](int s) { return bar0 + 8 * (14 + s); };
+    auto kv_full = [&](int st) { return bar0 + 8 * (16 + st); };
+    auto kv_empty = [&](int st) { return bar0 + 8 * (16 + kStages + st); };
     __shared__ uint32_t tmem_base_sh;
     __shared__ volatile int abort_flag;
 
@@ -213,10 +221,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
 
     if (tid == 0) {
         for (int s = 0; s < 2; ++s) {
-            mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1); mbar_init(s_full(s), 1);
-            mbar_init(p_full(s), 4); mbar_init(o_done(s), 1);   // p_full: one arrival per softmax warp
+            mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1);
+            mbar_init(s_full(s, 0), 1); mbar_init(s_full(s, 1), 1);
+            mbar_init(p_full(s, 0), 4); mbar_init(p_full(s, 1), 4);   // one arrival per softmax warp
+            mbar_init(pv_done(s), 1); mbar_init(o_done(s), 1);
         }
-        for (int st = 0; st < kStages; ++st) { mbar_init(kv_full(st), 1); mbar_init(kv_empty(st), 1); }
+        for (int st = 0; st < kStages; ++st) {
+            mbar_init(kv_full(st), 1);
+            mbar_init(kv_empty(st), 2);                 // both issuers release a stage
+        }
         abort_flag = 0;
         fence_barrier_init();
     }
@@ -232,10 +245,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     };
 
     if (warp >= 8) {
-    // register budget: this warpgroup gives registers up, the softmax warpgroups (which hold a
-    // whole S row per thread) take them
+    // register budget: this warpgroup gives registers up, the softmax warpgroups take them
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLow));
-    if (warp == 9) {
+    if (warp == 11) {
+        // idle
+    } else if (warp == 9) {
         // ------------------------------------------------------------------ TMA loader
         if (elect_one()) {
             prefetch_tmap(&mQ); prefetch_tmap(&mKc); prefetch_tmap(&mVc);
@@ -250,9 +264,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                     const uint32_t qc = s ? qcnt1 : qcnt0;
                     if (abort_flag || !mbar_wait(q_empty(s), (qc & 1u) ^ 1u)) { fail(100); ok = false; break; }
                     if (s) ++qcnt1; else ++qcnt0;
-                    mbar_arrive_expect_tx(q_full(s), kTileBytes);
-                    tma_load_3d(sQ + s * kTileBytes, &mQ, q_full(s), 0, g.head, qrow + s * kBM);
-                    tma_load_3d(sQ + s * kTileBytes + kHalfBytes, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
+                    mbar_arrive_expect_tx(q_full(s), kQBytes);
+                    tma_load_3d(sQ + s * kQBytes, &mQ, q_full(s), 0, g.head, qrow + s * kBM);
+                    tma_load_3d(sQ + s * kQBytes + kQHalf, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
                 }
                 for (int j = g.t0; j < g.t1 && ok; ++j) {
                     const bool seg2 = j >= g.nt1;
@@ -276,74 +290,104 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
             }
         }
         __syncwarp();
-    } else if (warp == 8) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else {
+        // ------------------------------------- MMA issuers: warp 8 -> slot 0, warp 10 -> slot 1
         if (elect_one()) {
+            const int slot = warp == 8 ? 0 : 1;
             const uint32_t idesc_qk = make_idesc_bf16(kBM, kBN, false, false);
             const uint32_t idesc_pv = make_idesc_bf16(kBM, kD, false, true);
             // Descriptors differ from tile to tile only in the 14-bit start-address field, so the
             // constant part is built once and the address (in 16-byte units) is added per MMA.
             const uint64_t desc_k = make_smem_desc_sw128(0, 16, 1024);             // K-major Q / K
             const uint64_t desc_v = make_smem_desc_sw128(0, kHalfBytes, 1024);     // MN-major V
-            auto issue_qk = [&](int slot, int stage) {
-                const uint64_t a = desc_k + ((sQ + slot * kTileBytes) >> 4);
+            const uint64_t desc_q = desc_k + ((sQ + slot * kQBytes) >> 4);
+            const uint32_t tSslot = tmem + slot * 128;
+            const uint32_t tOslot = tmem + 256 + slot * kD;
+            auto issue_qk = [&](int buf, int stage) {          // S[buf] = Q K^T, N = 64 keys
                 const uint64_t b = desc_k + ((sKV + stage * kTileBytes) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < kD / 16; ++kk) {
-                    const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
-                    umma_ss(tmem + slot * kBN, a + off, b + off, idesc_qk, kk > 0);
+                    const uint32_t qoff = ((kk >> 2) * kQHalf + (kk & 3) * 32) >> 4;
+                    const uint32_t koff = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+                    umma_ss(tSslot + buf * kBN, desc_q + qoff, b + koff, idesc_qk, kk > 0);
                 }
             };
-            auto issue_pv = [&](int slot, int stage, bool first) {
+            auto issue_pv = [&](int buf, int stage, bool first) {   // O += P[buf] V, K = 64 keys
                 const uint64_t b = desc_v + ((sKV + stage * kTileBytes) >> 4);
 #pragma unroll
                 for (int kk = 0; kk < kBN / 16; ++kk)
-                    umma_ts(tmem + 256 + slot * kD, tmem + slot * kBN + kk * 8, b + kk * (2048 >> 4), idesc_pv,
+                    umma_ts(tOslot, tSslot + buf * kBN + kk * 8, b + kk * (2048 >> 4), idesc_pv,
                             !(first && kk == 0));
             };
+            // The issuing thread shares its scheduler with two softmax warps, so its own
+            // instruction count per tile matters: ring positions are advanced incrementally (no
+            // division), and the abort flag is only looked at when a wait fails.
             bool ok = true;
             auto wait = [&](uint32_t bar, uint32_t ph, int code) {
-                if (!ok) return;
-                if (abort_flag || !mbar_wait(bar, ph)) { fail(code); ok = false; }
+                if (!mbar_wait(bar, ph)) { fail(code); ok = false; }
+            };
+            struct Cursor {                      // position of a ring entry: stage and phase bit
+                uint32_t st, ph;
+                __device__ __forceinline__ void step(uint32_t k) {
+                    st += k;
+                    if (st >= (uint32_t)kStages) { st -= kStages; ph ^= 1u; }
+                }
             };
             SegIter iter(p, blockIdx.x, gridDim.x);
             Seg g;
-            uint32_t ring = 0, qcnt0 = 0, qcnt1 = 0, pcnt0 = 0, pcnt1 = 0;
+            Cursor cur{0u, 0u};                  // first ring entry of the next run
+            uint32_t qcnt = 0, tc = 0;           // tc: tiles this slot has processed so far
             while (ok && iter.next(p, g)) {
-                for (int s = 0; s < g.n_slots; ++s) {
-                    wait(q_full(s), (s ? qcnt1 : qcnt0) & 1u, 201);
-                    if (s) ++qcnt1; else ++qcnt0;
+                const int n = g.t1 - g.t0;
+                if (slot >= g.n_slots) {
+                    // nothing to compute for this slot, but every K/V stage is released by both issuers
+                    for (int e = 0; e < 2 * n && ok; ++e) {
+                        wait(kv_full(cur.st), cur.ph, 206);
+                        if (ok) mbar_arrive(kv_empty(cur.st));
+                        cur.step(1);
+                    }
+                    continue;
                 }
-                {   // S(t0) for every live slot
-                    const int st = ring % kStages;
-                    wait(kv_full(st), (ring / kStages) & 1u, 202);
+                wait(q_full(slot), qcnt & 1u, 201);
+                ++qcnt;
+                // ring entries of this run: K_i at +2i, V_i at +2i+1
+                Cursor ck = cur, cv = cur;
+                cv.step(1);
+                for (int i = 0; i < 2 && i < n && ok; ++i) {        // S(0), S(1)
+                    wait(kv_full(ck.st), ck.ph, 202);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    for (int s = 0; s < g.n_slots; ++s) { issue_qk(s, st); umma_commit(s_full(s)); }
-                    umma_commit(kv_empty(st));
-                    ++ring;
+                    issue_qk((tc + i) & 1, ck.st);
+                    umma_commit(s_full(slot, (tc + i) & 1));
+                    umma_commit(kv_empty(ck.st));
+                    ck.step(2);
                 }
-                for (int j = g.t0; j < g.t1 && ok; ++j) {
-                    const bool more = j + 1 < g.t1;
-                    const uint32_t rv = ring, rk = ring + 1;           // V_j and K_{j+1}
-                    const int stv = rv % kStages, stk = rk % kStages;
-                    wait(kv_full(stv), (rv / kStages) & 1u, 203);
-                    if (more) wait(kv_full(stk), (rk / kStages) & 1u, 204);
-                    for (int s = 0; s < g.n_slots && ok; ++s) {
-                        if (ok && (abort_flag || !mbar_wait_spin(p_full(s), (s ? pcnt1 : pcnt0) & 1u))) { fail(205); ok = false; }
+                if (n == 1) ck.step(2);                              // keep ck two tiles ahead of cv
+#pragma unroll 1
+                for (int i = 0; i < n && ok; ++i) {
+                    const int buf = (tc + i) & 1;
+                    wait(kv_full(cv.st), cv.ph, 203);
+                    if (!ok) break;
+                    if (!mbar_wait_spin(p_full(slot, buf), ((tc + i) >> 1) & 1u)) { fail(205); ok = false; break; }
+                    tc_fence_after_sync();
+                    issue_pv(buf, cv.st, i == 0);
+                    umma_commit(kv_empty(cv.st));
+                    if (i + 2 < n) {                                // S(i+2) reuses the buffer P(i) was read from
+                        wait(kv_full(ck.st), ck.ph, 204);
                         if (!ok) break;
-                        if (s) ++pcnt1; else ++pcnt0;
-                        tc_fence_after_sync();
-                        issue_pv(s, stv, j == g.t0);
-                        if (more) { issue_qk(s, stk); umma_commit(s_full(s)); }
-                        else { umma_commit(o_done(s)); umma_commit(q_empty(s)); }
+                        issue_qk(buf, ck.st);
+                        umma_commit(s_full(slot, buf));
+                        umma_commit(kv_empty(ck.st));
+                    } else if (i + 2 == n) {
+                        umma_commit(pv_done(slot));                 // lets the last tile's softmax know O is at rest
                     }
-                    if (ok) {
-                        umma_commit(kv_empty(stv));
-                        if (more) umma_commit(kv_empty(stk));
-                    }
-                    ring += more ? 2 : 1;
+                    if (i == n - 1) { umma_commit(o_done(slot)); umma_commit(q_empty(slot)); }
+                    cv.step(2);
+                    ck.step(2);
                 }
+                tc += (uint32_t)n;
+                cur.step((2u * (uint32_t)n) % kStages);
+                if (((2u * (uint32_t)n) / kStages) & 1u) cur.ph ^= 1u;
             }
         }
         __syncwarp();
@@ -354,60 +398,62 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
         const int slot = warp >> 2;
         const int row_in_slot = tid & 127;
         const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
-        const uint32_t tS = tmem + slot * kBN + lane_base;
+        const uint32_t tSslot = tmem + slot * 128 + lane_base;
         const uint32_t tO = tmem + 256 + slot * kD + lane_base;
         const float sl2 = p.scale * 1.4426950408889634f;
+        const uint64_t sl2_2 = pack2(__float_as_uint(sl2), __float_as_uint(sl2));
         SegIter iter(p, blockIdx.x, gridDim.x);
         Seg g;
-        uint32_t scnt = 0, ocnt = 0;
+        uint32_t tc = 0, ocnt = 0, pvcnt = 0;     // pvcnt: runs of two or more tiles so far
         bool ok = true;
         while (ok && iter.next(p, g)) {
             if (slot >= g.n_slots) continue;
             float m_used = -INFINITY, l_sum = 0.f;
-            for (int j = g.t0; j < g.t1; ++j) {
+            const int n = g.t1 - g.t0;
+            for (int i = 0; i < n; ++i) {
+                const int j = g.t0 + i;
+                const int buf = (tc + i) & 1;
+                const uint32_t tS = tSslot + buf * kBN;
                 {
-                    const bool w = mbar_wait_spin(s_full(slot), scnt & 1u) && !abort_flag;
+                    const bool w = mbar_wait_spin(s_full(slot, buf), ((tc + i) >> 1) & 1u) && !abort_flag;
                     if (!__all_sync(0xffffffffu, w)) { fail(301); ok = false; break; }   // warp-uniform
-                    ++scnt;
                 }
                 tc_fence_after_sync();
-                uint32_t sr[128];
+                uint32_t sr[64];
                 const bool seg2 = j >= g.nt1;
                 const int64_t left = (seg2 ? g.nC - (int64_t)(j - g.nt1) * kBN : g.nB - (int64_t)j * kBN);
-                const float sl2n = sl2;
-                const uint64_t sl2_2 = pack2(__float_as_uint(sl2n), __float_as_uint(sl2n));
                 // Fast path (every tile but a run's first and a segment's ragged last): the
                 // exponentials use the running maximum as it stands, so they start as soon as
-                // the first quarter of S has arrived and overlap the remaining TMEM loads; the
-                // tile's own maximum is only needed for the (rare) rescale decision at the end.
-                bool full_pass = (j == g.t0) || (left < kBN);
+                // the first half of S has arrived; the tile's own maximum only feeds the (rare)
+                // rescale decision at the end.
+                bool full_pass = (i == 0) || (left < kBN);
                 if (!full_pass) {
                     const float mbf = -m_used * sl2;
                     const uint64_t mb_2 = pack2(__float_as_uint(mbf), __float_as_uint(mbf));
                     uint64_t rs2[2] = {0ull, 0ull};
-                    float mx4[4];
+                    float mx2[2];
                     PAFU_TMEM_LD_X32(tS, sr);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (c < 3) PAFU_TMEM_LD_X32(tS + 32 * (c + 1), sr + 32 * (c + 1));
+                    for (int c = 0; c < 2; ++c) {
+                        if (c == 0) PAFU_TMEM_LD_X32(tS + 32, sr + 32);
                         uint32_t pk[16];
                         float m = -INFINITY;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const uint32_t u0 = sr[32 * c + 2 * i], u1 = sr[32 * c + 2 * i + 1];
+                        for (int q = 0; q < 16; ++q) {
+                            const uint32_t u0 = sr[32 * c + 2 * q], u1 = sr[32 * c + 2 * q + 1];
                             float e0, e1;
                             unpack2(ffma2(pack2(u0, u1), sl2_2, mb_2), e0, e1);
                             const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
-                            rs2[i & 1] = fadd2(rs2[i & 1], pack2(__float_as_uint(p0), __float_as_uint(p1)));
-                            pk[i] = pack_bf16(p0, p1);
+                            rs2[q & 1] = fadd2(rs2[q & 1], pack2(__float_as_uint(p0), __float_as_uint(p1)));
+                            pk[q] = pack_bf16(p0, p1);
                             m = fmax3(m, __uint_as_float(u0), __uint_as_float(u1));
                         }
-                        mx4[c] = m;
+                        mx2[c] = m;
                         PAFU_TMEM_ST_X16(tS + 16 * c, pk);
-                        if (c < 3) tmem_wait_ld();
+                        if (c == 0) tmem_wait_ld();
                     }
-                    const float mxf = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                    const float mxf = fmaxf(mx2[0], mx2[1]);
                     full_pass = __any_sync(0xffffffffu, (mxf - m_used) * sl2 > kRescaleThresholdLog2);
                     if (!full_pass) {
                         float r0, r1, r2, r3;
@@ -418,75 +464,75 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 } else {
                     PAFU_TMEM_LD_X32(tS, sr);
                     PAFU_TMEM_LD_X32(tS + 32, sr + 32);
-                    PAFU_TMEM_LD_X32(tS + 64, sr + 64);
-                    PAFU_TMEM_LD_X32(tS + 96, sr + 96);
                     tmem_wait_ld();
                     if (left < kBN) {          // ragged end of a key segment
 #pragma unroll
-                        for (int c = 0; c < 128; ++c)
+                        for (int c = 0; c < kBN; ++c)
                             if (c >= left) sr[c] = 0xff800000u;   // -inf
                     }
                 }
                 if (full_pass) {
-                // row maximum: four independent chains of 3-input max
-                float mx4[4];
+                    float mx4[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    float m = fmaxf(__uint_as_float(sr[32 * q]), __uint_as_float(sr[32 * q + 1]));
+                    for (int q = 0; q < 4; ++q) {
+                        float m = fmaxf(__uint_as_float(sr[16 * q]), __uint_as_float(sr[16 * q + 1]));
 #pragma unroll
-                    for (int c = 2; c < 32; c += 2)
-                        m = fmax3(m, __uint_as_float(sr[32 * q + c]), __uint_as_float(sr[32 * q + c + 1]));
-                    mx4[q] = m;
-                }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                if (j == g.t0) {
-                    m_used = mx;
-                } else if (__any_sync(0xffffffffu, (mx - m_used) * sl2 > kRescaleThresholdLog2)) {
-                    // the whole warp rescales together (TMEM accesses are warp-collective);
-                    // rows whose maximum did not move get alpha = 1
-                    const float m_new = fmaxf(m_used, mx);
-                    const float alpha = fast_exp2((m_used - m_new) * sl2);
-                    l_sum *= alpha;
-                    m_used = m_new;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t orr[32];
-                        PAFU_TMEM_LD_X32(tO + c * 32, orr);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) orr[i] = __float_as_uint(__uint_as_float(orr[i]) * alpha);
-                        PAFU_TMEM_ST_X32(tO + c * 32, orr);
+                        for (int c = 2; c < 16; c += 2)
+                            m = fmax3(m, __uint_as_float(sr[16 * q + c]), __uint_as_float(sr[16 * q + c + 1]));
+                        mx4[q] = m;
                     }
-                }
-                // p = 2^(s * sl2 - m * sl2): packed FMA for the exponent, packed adds for the sum
-                const float mb = -m_used * sl2;
-                const uint64_t mb_2 = pack2(__float_as_uint(mb), __float_as_uint(mb));
-                uint64_t rs2[2] = {0ull, 0ull};
+                    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                    if (i == 0) {
+                        m_used = mx;
+                    } else if (__any_sync(0xffffffffu, (mx - m_used) * sl2 > kRescaleThresholdLog2)) {
+                        // The whole warp rescales together (TMEM accesses are warp-collective); rows
+                        // whose maximum did not move get alpha = 1.  O must be at rest, i.e. the previous
+                        // tile's P V product finished: S(i+1) being ready implies it (it was issued
+                        // after that product); the run's last tile has a barrier of its own.
+                        const bool w = (i + 1 < n ? mbar_wait(s_full(slot, buf ^ 1), ((tc + i + 1) >> 1) & 1u)
+                                                  : mbar_wait(pv_done(slot), pvcnt & 1u)) && !abort_flag;
+                        if (!__all_sync(0xffffffffu, w)) { fail(303); ok = false; break; }
+                        tc_fence_after_sync();
+                        const float m_new = fmaxf(m_used, mx);
+                        const float alpha = fast_exp2((m_used - m_new) * sl2);
+                        l_sum *= alpha;
+                        m_used = m_new;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t orr[32];
+                            PAFU_TMEM_LD_X32(tO + c * 32, orr);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int q = 0; q < 32; ++q) orr[q] = __float_as_uint(__uint_as_float(orr[q]) * alpha);
+                            PAFU_TMEM_ST_X32(tO + c * 32, orr);
+                        }
+                    }
+                    const float mb = -m_used * sl2;
+                    const uint64_t mb_2 = pack2(__float_as_uint(mb), __float_as_uint(mb));
+                    uint64_t rs2[2] = {0ull, 0ull};
                     uint32_t pk[32];
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
                         float e0, e1;
-                        unpack2(ffma2(pack2(sr[64 * h + 2 * c], sr[64 * h + 2 * c + 1]), sl2_2, mb_2), e0, e1);
+                        unpack2(ffma2(pack2(sr[2 * c], sr[2 * c + 1]), sl2_2, mb_2), e0, e1);
                         const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
                         rs2[c & 1] = fadd2(rs2[c & 1], pack2(__float_as_uint(p0), __float_as_uint(p1)));
                         pk[c] = pack_bf16(p0, p1);
                     }
-                    PAFU_TMEM_ST_X32(tS + 32 * h, pk);
-                }
-                float r0, r1, r2, r3;
-                unpack2(rs2[0], r0, r1);
-                unpack2(rs2[1], r2, r3);
-                const float rs = (r0 + r1) + (r2 + r3);
-                l_sum += rs;
+                    PAFU_TMEM_ST_X32(tS, pk);
+                    float r0, r1, r2, r3;
+                    unpack2(rs2[0], r0, r1);
+                    unpack2(rs2[1], r2, r3);
+                    l_sum += (r0 + r1) + (r2 + r3);
                 }   // full_pass
                 tmem_wait_st();
                 tc_fence_before_sync();
                 __syncwarp();
-                if ((tid & 31) == 0) mbar_arrive(p_full(slot));
+                if ((tid & 31) == 0) mbar_arrive(p_full(slot, buf));
             }
             if (!ok) break;
+            tc += (uint32_t)n;
+            if (n >= 2) ++pvcnt;
             {
                 const bool w = mbar_wait(o_done(slot), ocnt & 1u) && !abort_flag;
                 if (!__all_sync(0xffffffffu, w)) { fail(302); ok = false; break; }
