@@ -55,6 +55,7 @@ constexpr int kTileBytes = kBN * kD * 2;      // 16 KiB: one K or V tile
 constexpr int kHalfBytes = kTileBytes / 2;    // one [64 rows x 64 cols] swizzled half
 constexpr int kSmemBytes = 2 * kQBytes + kStages * kTileBytes + 1024 /*align*/ + 512 /*barriers*/;
 constexpr float kRescaleThresholdLog2 = 8.0f;
+constexpr float kSumTrigger = 65536.0f;   // a 64-key row sum this large means some p exceeded 2^10
 // Register re-balancing.  With 384 threads the kernel launches with 168 registers per thread.
 // setmaxnreg.inc blocks until the registers exist, so what the third warpgroup gives up must
 // cover what the two softmax warpgroups take: (168 - kRegsLow) * 128 >= (kRegsHigh - 168) * 256.
@@ -410,66 +411,55 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
             if (slot >= g.n_slots) continue;
             float m_used = -INFINITY, l_sum = 0.f;
             const int n = g.t1 - g.t0;
+            uint32_t sr[64];
+            bool loaded = false;                       // S(i) already requested from tensor memory
             for (int i = 0; i < n; ++i) {
                 const int j = g.t0 + i;
                 const int buf = (tc + i) & 1;
                 const uint32_t tS = tSslot + buf * kBN;
-                {
+                if (!loaded) {
                     const bool w = mbar_wait_spin(s_full(slot, buf), ((tc + i) >> 1) & 1u) && !abort_flag;
                     if (!__all_sync(0xffffffffu, w)) { fail(301); ok = false; break; }   // warp-uniform
+                    tc_fence_after_sync();
+                    PAFU_TMEM_LD_X32(tS, sr);
+                    PAFU_TMEM_LD_X32(tS + 32, sr + 32);
                 }
-                tc_fence_after_sync();
-                uint32_t sr[64];
+                loaded = false;
+                tmem_wait_ld();
                 const bool seg2 = j >= g.nt1;
                 const int64_t left = (seg2 ? g.nC - (int64_t)(j - g.nt1) * kBN : g.nB - (int64_t)j * kBN);
                 // Fast path (every tile but a run's first and a segment's ragged last): the
-                // exponentials use the running maximum as it stands, so they start as soon as
-                // the first half of S has arrived; the tile's own maximum only feeds the (rare)
-                // rescale decision at the end.
+                // exponentials use the running maximum as it stands.  Only when the tile's row sum
+                // shows that some logit outgrew that maximum by more than 2^10 does the tile take
+                // the full pass below (true maximum, rescale of O and of the row sum).
                 bool full_pass = (i == 0) || (left < kBN);
                 if (!full_pass) {
                     const float mbf = -m_used * sl2;
                     const uint64_t mb_2 = pack2(__float_as_uint(mbf), __float_as_uint(mbf));
                     uint64_t rs2[2] = {0ull, 0ull};
-                    float mx2[2];
-                    PAFU_TMEM_LD_X32(tS, sr);
-                    tmem_wait_ld();
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
-                        if (c == 0) PAFU_TMEM_LD_X32(tS + 32, sr + 32);
                         uint32_t pk[16];
-                        float m = -INFINITY;
 #pragma unroll
                         for (int q = 0; q < 16; ++q) {
-                            const uint32_t u0 = sr[32 * c + 2 * q], u1 = sr[32 * c + 2 * q + 1];
                             float e0, e1;
-                            unpack2(ffma2(pack2(u0, u1), sl2_2, mb_2), e0, e1);
+                            unpack2(ffma2(pack2(sr[32 * c + 2 * q], sr[32 * c + 2 * q + 1]), sl2_2, mb_2), e0, e1);
                             const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
                             rs2[q & 1] = fadd2(rs2[q & 1], pack2(__float_as_uint(p0), __float_as_uint(p1)));
                             pk[q] = pack_bf16(p0, p1);
-                            m = fmax3(m, __uint_as_float(u0), __uint_as_float(u1));
                         }
-                        mx2[c] = m;
                         PAFU_TMEM_ST_X16(tS + 16 * c, pk);
-                        if (c == 0) tmem_wait_ld();
                     }
-                    const float mxf = fmaxf(mx2[0], mx2[1]);
-                    full_pass = __any_sync(0xffffffffu, (mxf - m_used) * sl2 > kRescaleThresholdLog2);
-                    if (!full_pass) {
-                        float r0, r1, r2, r3;
-                        unpack2(rs2[0], r0, r1);
-                        unpack2(rs2[1], r2, r3);
-                        l_sum += (r0 + r1) + (r2 + r3);
-                    }
-                } else {
-                    PAFU_TMEM_LD_X32(tS, sr);
-                    PAFU_TMEM_LD_X32(tS + 32, sr + 32);
-                    tmem_wait_ld();
-                    if (left < kBN) {          // ragged end of a key segment
+                    float r0, r1, r2, r3;
+                    unpack2(rs2[0], r0, r1);
+                    unpack2(rs2[1], r2, r3);
+                    const float rs = (r0 + r1) + (r2 + r3);
+                    full_pass = __any_sync(0xffffffffu, !(rs < kSumTrigger));    // also true for inf / NaN
+                    if (!full_pass) l_sum += rs;
+                } else if (left < kBN) {               // ragged end of a key segment
 #pragma unroll
-                        for (int c = 0; c < kBN; ++c)
-                            if (c >= left) sr[c] = 0xff800000u;   // -inf
-                    }
+                    for (int c = 0; c < kBN; ++c)
+                        if (c >= left) sr[c] = 0xff800000u;   // -inf
                 }
                 if (full_pass) {
                     float mx4[4];
@@ -525,6 +515,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                     unpack2(rs2[1], r2, r3);
                     l_sum += (r0 + r1) + (r2 + r3);
                 }   // full_pass
+                if (i + 1 < n && __all_sync(0xffffffffu, mbar_test_wait(s_full(slot, buf ^ 1), ((tc + i + 1) >> 1) & 1u))) {
+                    // S(i+1) is already complete: request it now, so that its trip from tensor
+                    // memory overlaps the hand-over of P(i)
+                    tc_fence_after_sync();
+                    PAFU_TMEM_LD_X32(tSslot + (buf ^ 1) * kBN, sr);
+                    PAFU_TMEM_LD_X32(tSslot + (buf ^ 1) * kBN + 32, sr + 32);
+                    loaded = true;
+                }
                 tmem_wait_st();
                 tc_fence_before_sync();
                 __syncwarp();
