@@ -2,14 +2,17 @@
 // Sec. 4.1): kept = [0, n_sink) U top-k salient of the middle U [T - n_recent, T), written as
 // ascending token indices, ties to the lower index.
 //
-// The step moves a few hundred KB, so it is latency-bound: one CTA of 1024 threads per
-// stream, scores read from L2 (once, into registers, when the stream is small enough).
+// The step moves a few hundred KB, so it is latency-bound: a cluster of eight CTAs per stream
+// with the candidates in registers (streams up to 32768 candidates), one CTA re-reading L2
+// for longer streams.
 //   1. fp32 scores map to order-preserving 32-bit keys (-0 folded onto +0, NaN lowest).
 //   2. MSB-first radix select (4 passes of 8 bits, shared-memory histograms) finds the key of
 //      the k-th largest candidate and how many candidates equal to it are still needed.
 //   3. Ordered emission: each thread owns a contiguous token range; two block-wide exclusive
 //      scans (ties seen so far, tokens kept so far) give every kept token its output slot,
 //      so the result is ascending and ties resolve to the lowest indices.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace pafu {
@@ -51,28 +54,38 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
     return warp_sums[warp] + inc - v;
 }
 
-constexpr int kSelRows = 32;                          // candidates per thread held in registers
-constexpr int kSelRegCap = kSelRows * kSelThreads;    // 32768 candidates
-constexpr int kSelList = 2048;                        // survivors of the first pass kept in shared memory
+constexpr int kSelCluster = 8;                        // CTAs cooperating on one stream
+constexpr int kSelRows = 4;                           // candidates per thread held in registers
+constexpr int kSelPerCta = kSelRows * kSelThreads;    // 4096
+constexpr int kSelRegCap = kSelCluster * kSelPerCta;  // 32768 candidates
 
-// Streams with at most kSelRegCap candidates: every candidate key is loaded once (all loads in
-// flight together) and stays in registers for the three radix passes (12 + 10 + 10 bits) and
-// the emission.  Candidate j of the stream sits in row j / 1024 of thread j % 1024, so a warp
-// ballot per row plus one block scan over the 32 x 32 (row, warp) counts gives every kept
-// candidate its ascending output slot.
+// Streams with at most kSelRegCap candidates: a cluster of eight CTAs per stream.  Candidate j
+// lives in CTA j / 4096, row (j / 1024) % 4, thread j % 1024, loaded once and kept in registers.
+// Every radix pass (12 + 10 + 10 bits) builds one shared-memory histogram per CTA; CTA r then
+// sums slice r of the bins over all eight histograms through distributed shared memory, the
+// slice totals are exchanged, and the CTA whose slice holds the k-th largest key finds the bin
+// and tells the others.  Emission: warp ballots per row, one block scan over the 4 x 32
+// (row, warp) counts, and the CTA totals exchanged through distributed shared memory give every
+// kept candidate its ascending output slot.
 __global__ void __launch_bounds__(kSelThreads)
-select_regs_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __restrict__ idx) {
+select_cluster_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __restrict__ idx) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
     __shared__ int hist[4096];
+    __shared__ int red[512];              // this CTA's slice of the cluster-wide histogram
+    __shared__ int slice_tot[kSelCluster];
+    __shared__ int cta_cnt[2][kSelCluster];   // per-CTA tie counts / keep counts
     __shared__ int cnt[kSelRows * 32];
-    __shared__ uint32_t list[kSelList];
     __shared__ int warp_sums[33];
     __shared__ uint32_t sh_prefix;
-    __shared__ int sh_krem, sh_bin, sh_nlist;
+    __shared__ int sh_krem, sh_bin;
 
-    const int s = blockIdx.x;
+    const int s = blockIdx.x / kSelCluster;
+    const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t T64 = st.cu_T[s + 1] - st.cu_T[s];
     const int64_t B64 = st.cu_B[s + 1] - st.cu_B[s];
+    // cluster-uniform exits (before any cluster barrier)
     if (B64 >= T64) return;                               // the streaming kernel writes the identity
     const int T = (int)T64;
     const int ns = (int)st.n_sink[s], nr = (int)st.n_recent[s];
@@ -81,16 +94,17 @@ select_regs_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __
     if (M > kSelRegCap) return;                           // the streaming kernel owns this stream
     const float* sc = scores + st.cu_T[s] + c0;
     int32_t* out = idx + st.cu_B[s];
+    const int j0 = rank * kSelPerCta;
 
     uint32_t key[kSelRows];
 #pragma unroll
     for (int i = 0; i < kSelRows; ++i) {
-        const int j = i * kSelThreads + tid;
+        const int j = j0 + i * kSelThreads + tid;
         key[i] = (j < M) ? score_key(__ldg(sc + j)) : 0u;
     }
-    // sink and recent tokens are kept as they are
-    for (int t = tid; t < ns; t += kSelThreads) out[t] = t;
-    for (int t = tid; t < nr; t += kSelThreads) out[ns + k + t] = T - nr + t;
+    // sink and recent tokens are kept as they are (spread over the cluster)
+    for (int t = rank * kSelThreads + tid; t < ns; t += kSelCluster * kSelThreads) out[t] = t;
+    for (int t = rank * kSelThreads + tid; t < nr; t += kSelCluster * kSelThreads) out[ns + k + t] = T - nr + t;
 
     uint32_t thr = 0xffffffffu;
     int need_eq = 0, eq_total = 0;
@@ -98,77 +112,78 @@ select_regs_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __
         uint32_t prefix = 0u, mask = 0u;
         int k_rem = k;
         int shift = 32;
-        int n_list = -1;                                  // >= 0: survivors are in list[]
 #pragma unroll 1
         for (int pass = 0; pass < 3; ++pass) {
             const int bits = pass == 0 ? 12 : 10;
             const int nb = 1 << bits;
+            const int slice = nb / kSelCluster;           // 512 or 128 bins per CTA
             shift -= bits;
             for (int b = tid; b < nb; b += kSelThreads) hist[b] = 0;
             __syncthreads();
-            if (n_list >= 0) {
-                // few candidates share the leading digit(s): work on the compacted list
-                for (int j = tid; j < n_list; j += kSelThreads) {
-                    const uint32_t kv = list[j];
-                    if ((kv & mask) == prefix) atomicAdd(&hist[(kv >> shift) & (uint32_t)(nb - 1)], 1);
-                }
-            } else {
 #pragma unroll
-                for (int i = 0; i < kSelRows; ++i) {
-                    const bool in = (i * kSelThreads + tid < M) && ((key[i] & mask) == prefix);
-                    const uint32_t digit = (key[i] >> shift) & (uint32_t)(nb - 1);
-                    // a warp whose live lanes all hold one digit (equal or saturated scores) adds once
-                    const unsigned act = __ballot_sync(0xffffffffu, in);
-                    if (act != 0u) {
-                        const uint32_t d0 = __shfl_sync(0xffffffffu, digit, __ffs(act) - 1);
-                        const bool uniform = __all_sync(0xffffffffu, !in || digit == d0);
-                        if (uniform) { if (lane == __ffs(act) - 1) atomicAdd(&hist[d0], __popc(act)); }
-                        else if (in) atomicAdd(&hist[digit], 1);
-                    }
+            for (int i = 0; i < kSelRows; ++i) {
+                const bool in = (j0 + i * kSelThreads + tid < M) && ((key[i] & mask) == prefix);
+                const uint32_t digit = (key[i] >> shift) & (uint32_t)(nb - 1);
+                // a warp whose live lanes all hold one digit (equal or saturated scores) adds once
+                const unsigned act = __ballot_sync(0xffffffffu, in);
+                if (act != 0u) {
+                    const uint32_t d0 = __shfl_sync(0xffffffffu, digit, __ffs(act) - 1);
+                    const bool uniform = __all_sync(0xffffffffu, !in || digit == d0);
+                    if (uniform) { if (lane == __ffs(act) - 1) atomicAdd(&hist[d0], __popc(act)); }
+                    else if (in) atomicAdd(&hist[digit], 1);
                 }
             }
-            __syncthreads();
-            // thread t owns bins nb-1 - t*bpt ... downwards; the exclusive scan of the per-thread
-            // counts is the number of matching candidates in all higher bins
-            const int bpt = nb >= kSelThreads ? nb / kSelThreads : 1;
+            cluster.sync();                                // every CTA's histogram is complete
+            // slice `rank` of the bins, summed over the cluster
             int mine = 0;
-            if (tid * bpt < nb)
-                for (int i = 0; i < bpt; ++i) mine += hist[nb - 1 - (tid * bpt + i)];
+            if (tid < slice) {
+                const int b = rank * slice + tid;
+#pragma unroll
+                for (int c = 0; c < kSelCluster; ++c) mine += *cluster.map_shared_rank(&hist[b], c);
+                red[tid] = mine;
+            }
             int total;
-            int above = block_exclusive_scan(mine, warp_sums, &total);
-            if (tid * bpt < nb) {
-                for (int i = 0; i < bpt; ++i) {
-                    const int b = nb - 1 - (tid * bpt + i);
-                    const int c = hist[b];
-                    if (above < k_rem && k_rem <= above + c) {
-                        sh_prefix = prefix | ((uint32_t)b << shift);
-                        sh_krem = k_rem - above;
-                        sh_bin = c;
+            // within the slice, higher bins first: thread t holds bin slice-1-t for the scan below
+            const int mine_desc = (tid < slice) ? 0 : 0;
+            (void)mine_desc;
+            block_exclusive_scan(mine, warp_sums, &total);     // only the total is needed here
+            if (tid == 0) {
+#pragma unroll
+                for (int c = 0; c < kSelCluster; ++c) *cluster.map_shared_rank(&slice_tot[rank], c) = total;
+            }
+            cluster.sync();                                // slice totals and red[] visible
+            // which slice holds the k-th largest matching key (slices scanned from the top)
+            int above = 0, q = kSelCluster - 1;
+            for (; q > 0; --q) {
+                if (k_rem <= above + slice_tot[q]) break;
+                above += slice_tot[q];
+            }
+            if (rank == q) {
+                // find the bin inside this slice: descending order, exclusive scan of counts
+                const int v = (tid < slice) ? red[slice - 1 - tid] : 0;
+                int tt;
+                const int ab = above + block_exclusive_scan(v, warp_sums, &tt);
+                if (tid < slice && ab < k_rem && k_rem <= ab + v) {
+                    const uint32_t bin = (uint32_t)(rank * slice + slice - 1 - tid);
+                    const uint32_t np = prefix | (bin << shift);
+                    for (int c = 0; c < kSelCluster; ++c) {
+                        *cluster.map_shared_rank(&sh_prefix, c) = np;
+                        *cluster.map_shared_rank(&sh_krem, c) = k_rem - ab;
+                        *cluster.map_shared_rank(&sh_bin, c) = v;
                     }
-                    above += c;
                 }
             }
-            if (tid == 0) sh_nlist = 0;
-            __syncthreads();
+            cluster.sync();                                // the decision has reached every CTA
             prefix = sh_prefix;
             k_rem = sh_krem;
+            eq_total = sh_bin;                             // after the last pass: keys equal to thr
             mask |= (uint32_t)(nb - 1) << shift;
-            eq_total = sh_bin;                            // after the last pass: keys equal to thr
-            if (pass == 0 && sh_bin <= kSelList) {
-                // gather the candidates that share the winning leading digit
-#pragma unroll
-                for (int i = 0; i < kSelRows; ++i)
-                    if ((i * kSelThreads + tid < M) && ((key[i] & mask) == prefix))
-                        list[atomicAdd(&sh_nlist, 1)] = key[i];
-                __syncthreads();
-                n_list = sh_nlist;
-            }
         }
         thr = prefix;
         need_eq = k_rem;
     }
 
-    // ---- ordered emission.  First the ties: rank of every candidate equal to the threshold.
+    // ---- ordered emission
     const unsigned lt_mask = (1u << lane) - 1u;
     uint32_t keep_bits = 0u;
     int total;
@@ -176,31 +191,33 @@ select_regs_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __
         // every candidate equal to the threshold is taken: no tie to break
 #pragma unroll
         for (int i = 0; i < kSelRows; ++i)
-            if ((i * kSelThreads + tid < M) && k > 0 && key[i] >= thr) keep_bits |= 1u << i;
+            if ((j0 + i * kSelThreads + tid < M) && k > 0 && key[i] >= thr) keep_bits |= 1u << i;
     } else {
-        uint32_t eq_bits = 0u;                            // bit i: row i equals the threshold
+        uint32_t eq_bits = 0u;
 #pragma unroll
         for (int i = 0; i < kSelRows; ++i) {
-            const bool eq = (i * kSelThreads + tid < M) && key[i] == thr;
+            const bool eq = (j0 + i * kSelThreads + tid < M) && key[i] == thr;
             const unsigned b = __ballot_sync(0xffffffffu, eq);
             if (lane == 0) cnt[i * 32 + warp] = __popc(b);
             if (eq) eq_bits |= 1u << i;
         }
         __syncthreads();
-        {
-            const int v = cnt[tid];
-            const int ex = block_exclusive_scan(v, warp_sums, &total);
-            __syncthreads();
-            cnt[tid] = ex;
-        }
+        const int v = (tid < kSelRows * 32) ? cnt[tid] : 0;
+        const int ex = block_exclusive_scan(v, warp_sums, &total);
         __syncthreads();
+        if (tid < kSelRows * 32) cnt[tid] = ex;
+        if (tid == 0)
+            for (int c = 0; c < kSelCluster; ++c) *cluster.map_shared_rank(&cta_cnt[0][rank], c) = total;
+        cluster.sync();
+        int eq_before = 0;
+        for (int c = 0; c < rank; ++c) eq_before += cta_cnt[0][c];
 #pragma unroll
         for (int i = 0; i < kSelRows; ++i) {
-            const bool valid = i * kSelThreads + tid < M;
+            const bool valid = j0 + i * kSelThreads + tid < M;
             const bool eq = (eq_bits >> i) & 1u;
             const unsigned b = __ballot_sync(0xffffffffu, eq);
-            const int rank = cnt[i * 32 + warp] + __popc(b & lt_mask);
-            const bool keep = valid && (key[i] > thr || (eq && rank < need_eq));
+            const int rk = eq_before + cnt[i * 32 + warp] + __popc(b & lt_mask);
+            const bool keep = valid && (key[i] > thr || (eq && rk < need_eq));
             if (keep) keep_bits |= 1u << i;
         }
     }
@@ -212,18 +229,23 @@ select_regs_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __
     }
     __syncthreads();
     {
-        const int v = cnt[tid];
+        const int v = (tid < kSelRows * 32) ? cnt[tid] : 0;
         const int ex = block_exclusive_scan(v, warp_sums, &total);
         __syncthreads();
-        cnt[tid] = ex;
+        if (tid < kSelRows * 32) cnt[tid] = ex;
+        if (tid == 0)
+            for (int c = 0; c < kSelCluster; ++c) *cluster.map_shared_rank(&cta_cnt[1][rank], c) = total;
     }
-    __syncthreads();
+    cluster.sync();
+    int kept_before = 0;
+    for (int c = 0; c < rank; ++c) kept_before += cta_cnt[1][c];
 #pragma unroll
     for (int i = 0; i < kSelRows; ++i) {
         const bool keep = (keep_bits >> i) & 1u;
         const unsigned b = __ballot_sync(0xffffffffu, keep);
-        if (keep) out[ns + cnt[i * 32 + warp] + __popc(b & lt_mask)] = c0 + i * kSelThreads + tid;
+        if (keep) out[ns + kept_before + cnt[i * 32 + warp] + __popc(b & lt_mask)] = c0 + j0 + i * kSelThreads + tid;
     }
+    cluster.sync();      // no CTA may exit while another can still write into its shared memory
 }
 
 // Streams with more candidates than the register kernel holds: keys are re-read from L2 in
@@ -339,7 +361,21 @@ pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* i
         any_regs |= regs;
         any_stream |= !regs;
     }
-    if (any_regs) select_regs_kernel<<<st.n_streams, kSelThreads, 0, stream>>>(scores, st, idx);
+    if (any_regs) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(st.n_streams * kSelCluster));
+        cfg.blockDim = dim3(kSelThreads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kSelCluster;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, select_cluster_kernel, scores, st, idx) != cudaSuccess) return PAFU_ERR_CUDA;
+    }
     if (any_stream) select_stream_kernel<<<st.n_streams, kSelThreads, 0, stream>>>(scores, st, idx);
     return cuda_ok(cudaGetLastError());
 }
