@@ -74,6 +74,7 @@ attn_mma_kernel(const uint16_t* __restrict__ Q, const uint16_t* __restrict__ Kc,
                 const uint16_t* __restrict__ Vc, const uint16_t* __restrict__ Kq,
                 const uint16_t* __restrict__ Vq, StreamTable st, int n_heads, float scale,
                 uint16_t* __restrict__ O, float* __restrict__ LSE) {
+    grid_dep_wait();
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int kTileBytes = 64 * D * 2;
     const uint32_t sQ = smem_u32(smem);
@@ -249,12 +250,12 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
         constexpr int smem = 5 * 64 * 128 * 2;
         e = cudaFuncSetAttribute(attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return PAFU_ERR_CUDA;
-        attn_mma_kernel<128><<<grid, kThreads, smem, stream>>>(Q, Kc, Vc, Kq, Vq, st, n_heads, scale, O, LSE);
+        launch_dependent(attn_mma_kernel<128>, dim3(grid), dim3(kThreads), smem, stream, 1, Q, Kc, Vc, Kq, Vq, st, n_heads, scale, O, LSE);
     } else {
         constexpr int smem = 5 * 64 * 64 * 2;
         e = cudaFuncSetAttribute(attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return PAFU_ERR_CUDA;
-        attn_mma_kernel<64><<<grid, kThreads, smem, stream>>>(Q, Kc, Vc, Kq, Vq, st, n_heads, scale, O, LSE);
+        launch_dependent(attn_mma_kernel<64>, dim3(grid), dim3(kThreads), smem, stream, 1, Q, Kc, Vc, Kq, Vq, st, n_heads, scale, O, LSE);
     }
     return cuda_ok(cudaGetLastError());
 }

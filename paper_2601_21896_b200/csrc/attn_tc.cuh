@@ -239,6 +239,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_sh;
+    grid_dep_wait();          // set-up above is local; everything below reads or writes global memory
 
     auto fail = [&](int code) {
         abort_flag = 1;
@@ -594,6 +595,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
 constexpr int kMergeRows = 4;
 __global__ void __launch_bounds__(1024)
 attn_tc_merge_kernel(const __grid_constant__ Params p, int n_cta) {
+    grid_dep_wait();
     __shared__ int piece_cta[kMaxGrid];
     __shared__ int n_pieces_sh;
     const int b = blockIdx.x >> 1, slot = blockIdx.x & 1;
@@ -717,11 +719,11 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
     }
     int grid = grid_for(cost);
     if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;   // caller's scratch holds fewer partials
-    attn_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(mQ, mKc, mVc, mKq, mVq, p);
-    if (cudaGetLastError() != cudaSuccess) return PAFU_ERR_CUDA;
+    if (launch_dependent(attn_tc_kernel, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mKc, mVc, mKq, mVq, p) != cudaSuccess)
+        return PAFU_ERR_CUDA;
     if (grid > 1) {
-        attn_tc_merge_kernel<<<2 * grid, 1024, 0, stream>>>(p, grid);
-        if (cudaGetLastError() != cudaSuccess) return PAFU_ERR_CUDA;
+        if (launch_dependent(attn_tc_merge_kernel, dim3(2 * grid), dim3(1024), 0, stream, 1, p, grid) != cudaSuccess)
+            return PAFU_ERR_CUDA;
     }
     return PAFU_OK;
 }

@@ -42,6 +42,39 @@ inline int device_sm_count() {
     return n;
 }
 
+// Every kernel of this library is launched with programmatic stream serialization: its CTAs
+// may be scheduled, and run their local set-up, as soon as the preceding kernel's CTAs have
+// left the SMs, without waiting for that kernel's completion to be processed first.  In return
+// each kernel executes grid_dep_wait() before its first access to global memory; that wait
+// returns only when the preceding kernel has completed and its writes are visible.  No kernel
+// signals its dependents early: CTAs of a following kernel that sat on the SMs while a
+// bandwidth-bound kernel was still in its last wave cost more than the earlier start gained.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                    cudaStream_t stream, unsigned cluster_x, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 1;
+    if (cluster_x > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = cluster_x;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
+    cfg.attrs = attr;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Launchers (each enqueues on `stream` and returns the launch status).
 pafu_status launch_score(const pafu_head& head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
                          float* scores, void* ws, size_t ws_bytes, cudaStream_t stream);

@@ -24,6 +24,7 @@ compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
                     StreamTable st, int32_t chunks_per_row,
                     uint4* __restrict__ Kc, uint4* __restrict__ Vc, float* __restrict__ SLc,
                     int64_t n_rows) {
+    grid_dep_wait();
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = (int64_t)blockIdx.x * kCompactWarpsPerBlock + (threadIdx.x >> 5);
     const int64_t n_warps = (int64_t)gridDim.x * kCompactWarpsPerBlock;
@@ -61,10 +62,9 @@ pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL
     int64_t blocks = (n_rows + kCompactWarpsPerBlock - 1) / kCompactWarpsPerBlock;
     const int64_t max_blocks = 148 * 8 * 4;   // a few resident waves; larger inputs loop
     if (blocks > max_blocks) blocks = max_blocks;
-    compact_rows_kernel<<<(unsigned)blocks, kCompactWarpsPerBlock * 32, 0, stream>>>(
-        reinterpret_cast<const uint4*>(K), reinterpret_cast<const uint4*>(V), SL, idx, st, chunks,
-        reinterpret_cast<uint4*>(Kc), reinterpret_cast<uint4*>(Vc), SLc, n_rows);
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(launch_dependent(compact_rows_kernel, dim3((unsigned)blocks), dim3(kCompactWarpsPerBlock * 32), 0, stream, 1,
+                                    reinterpret_cast<const uint4*>(K), reinterpret_cast<const uint4*>(V), SL, idx, st,
+                                    chunks, reinterpret_cast<uint4*>(Kc), reinterpret_cast<uint4*>(Vc), SLc, n_rows));
 }
 
 }  // namespace pafu

@@ -102,6 +102,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
         fence_barrier_init();
     }
     if (warp == 8) { tmem_alloc(smem_u32(&tmem_base_sh), 512); tmem_relinquish(); }
+    grid_dep_wait();          // set-up above is local; everything below reads or writes global memory
     // folded second layer and first-layer bias, fp32 in shared memory
     for (int h = tid; h < p.d_hidden; h += kThreads) {
         float m = 0.f;
@@ -250,9 +251,9 @@ inline pafu_status launch(const pafu_head& head, const uint16_t* X, int64_t n_to
             return PAFU_ERR_CUDA;
         attr_set = true;
     }
-    if (head.act == PAFU_ACT_GELU) score_tc_kernel<PAFU_ACT_GELU><<<grid, kThreads, kSmemBytes, stream>>>(mX, mW, p);
-    else score_tc_kernel<PAFU_ACT_SILU><<<grid, kThreads, kSmemBytes, stream>>>(mX, mW, p);
-    return cuda_ok(cudaGetLastError());
+    return cuda_ok(head.act == PAFU_ACT_GELU
+                       ? launch_dependent(score_tc_kernel<PAFU_ACT_GELU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mX, mW, p)
+                       : launch_dependent(score_tc_kernel<PAFU_ACT_SILU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mX, mW, p));
 }
 
 }  // namespace score_tc

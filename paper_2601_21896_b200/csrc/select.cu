@@ -69,6 +69,7 @@ constexpr int kSelRegCap = kSelCluster * kSelPerCta;  // 32768 candidates
 // kept candidate its ascending output slot.
 __global__ void __launch_bounds__(kSelThreads)
 select_cluster_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __restrict__ idx) {
+    grid_dep_wait();
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ int hist[4096];
@@ -252,6 +253,7 @@ select_cluster_kernel(const float* __restrict__ scores, StreamTable st, int32_t*
 // every pass (4 passes of 8 bits), and each thread emits a contiguous token range.
 __global__ void __launch_bounds__(kSelThreads)
 select_stream_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __restrict__ idx) {
+    grid_dep_wait();
     if (st.cu_T[blockIdx.x + 1] - st.cu_T[blockIdx.x] - st.n_sink[blockIdx.x] - st.n_recent[blockIdx.x] <= kSelRegCap &&
         st.cu_B[blockIdx.x + 1] - st.cu_B[blockIdx.x] < st.cu_T[blockIdx.x + 1] - st.cu_T[blockIdx.x]) return;   // the register kernel owns this stream
     __shared__ int hist[256];
@@ -362,21 +364,14 @@ pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* i
         any_stream |= !regs;
     }
     if (any_regs) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(st.n_streams * kSelCluster));
-        cfg.blockDim = dim3(kSelThreads);
-        cfg.dynamicSmemBytes = 0;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = kSelCluster;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, select_cluster_kernel, scores, st, idx) != cudaSuccess) return PAFU_ERR_CUDA;
+        if (launch_dependent(select_cluster_kernel, dim3((unsigned)(st.n_streams * kSelCluster)), dim3(kSelThreads), 0,
+                             stream, kSelCluster, scores, st, idx) != cudaSuccess)
+            return PAFU_ERR_CUDA;
     }
-    if (any_stream) select_stream_kernel<<<st.n_streams, kSelThreads, 0, stream>>>(scores, st, idx);
+    if (any_stream &&
+        launch_dependent(select_stream_kernel, dim3((unsigned)st.n_streams), dim3(kSelThreads), 0, stream, 1, scores, st,
+                         idx) != cudaSuccess)
+        return PAFU_ERR_CUDA;
     return cuda_ok(cudaGetLastError());
 }
 
