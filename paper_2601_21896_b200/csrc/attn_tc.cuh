@@ -17,9 +17,10 @@
 //   warps 0-3  softmax of slot 0 (thread = query row = TMEM lane)
 //   warps 4-7  softmax of slot 1
 //   warps 8,10 MMA issuers, one per slot: S = Q K^T (both operands in shared memory) and
-//              O += P V (P read from tensor memory, V from shared memory, MN-major).  One thread
-//              can start a tcgen05.mma only about every 100 clocks while the tensor core
-//              finishes a 128x128x16 one in 64, hence an issuing thread per slot
+//              O += P V (P read from tensor memory, V from shared memory, MN-major).  With the
+//              waits, commits and descriptor arithmetic of its loop one thread sustains about
+//              one tcgen05.mma per 100 clocks while the tensor core finishes a 128x128x16 one
+//              in 64, hence an issuing thread per slot
 //   warp  9    TMA loader: Q tiles per item, 64-key K/V tiles through a 10-stage ring that
 //              runs ahead across item boundaries
 //   warp  11   idle (completes the third warpgroup so registers can be re-balanced)
