@@ -244,7 +244,7 @@ def run_ours(args):
     import torch.distributed as dist
     import paper_2601_21896_b200 as pafu
     from paper_2601_21896_b200 import workloads as wl
-    from paper_2601_21896_b200.harness import Layer
+    from paper_2601_21896_b200.harness import Layer, to_device_bf16
     from paper_2601_21896_b200 import sharding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -342,6 +342,38 @@ def run_ours(args):
     d2h = int(h_scores.numel() * 4 + h_idx.numel() * 4 + h_O.numel() * 2)
     e2e_value = world * work["attn_flops"] / (e2e_ms * 1e-3) / 1e12
 
+    # ---- the paper's own S-MLP on the new chunk (Appendix A: [q, k, v] -> 1024 -> 12, SiLU, mean),
+    # read from the chunk's Q / K / V in place.  Its 43 MB of inputs fit in L2, so a buffer larger
+    # than L2 is written between launches.
+    qkv = None
+    if rank == 0 and w.d_model % 64 == 0:
+        rng = np.random.default_rng(7)
+        d3, dh, do = 3 * w.d_model, 1024, 12
+        bits = lambda shape, sc: to_device_bf16(wl.f32_to_bf16_bits((rng.standard_normal(shape) * sc).astype(np.float32)))
+        phead = pafu.Head(bits((dh, d3), d3 ** -0.5), bits((dh,), 0.3), bits((do, dh), dh ** -0.5), bits((do,), 0.3),
+                          wl.ACT_SILU, wl.FINAL_NONE)
+        pws = torch.zeros(pafu.pafu_workspace_bytes(L0.shape, None, phead), dtype=torch.uint8, device="cuda")
+        pout = torch.empty(L0.nQ, dtype=torch.float32, device="cuda")
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        reps = 12
+        evq = [new_events(2) for _ in range(reps)]
+        for r in range(reps + 3):
+            flush.fill_(r & 1)
+            if r >= 3:
+                evq[r - 3][0].record(stream)
+            pafu.pafu_score_qkv(phead, L0.Q, L0.Kq, L0.Vq, pout, pws, n_tokens=L0.nQ, ld=w.d_model)
+            if r >= 3:
+                evq[r - 3][1].record(stream)
+        torch.cuda.synchronize()
+        assert pafu.pafu_workspace_status(pws) == 0
+        q_ms = float(np.median([a.elapsed_time(b) for a, b in evq]))
+        q_flops = 2.0 * L0.nQ * d3 * dh
+        q_bytes = L0.nQ * d3 * 2 + dh * d3 * 2 + L0.nQ * 4
+        qkv = {"workload": "paper S-MLP on the chunk: %d tokens, [q,k,v] %d -> %d -> %d, SiLU, mean" % (L0.nQ, d3, dh, do),
+               "ms": q_ms, "TFLOP/s": q_flops / (q_ms * 1e-3) / 1e12, "GB/s": q_bytes / (q_ms * 1e-3) / 1e9,
+               "l2": "256 MB written between launches"}
+        del flush
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -378,6 +410,7 @@ def run_ours(args):
                 "hbm_frac": gbs(work["score_bytes"] + work["select_bytes"] + work["compact_bytes"],
                                 k_ms[:3].sum()) / peaks["hbm_gbs"]},
         },
+        "score_qkv": qkv,
         "layers_per_step": n_layers,
         "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step / n_layers,
         "peaks": peaks,

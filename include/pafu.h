@@ -130,6 +130,16 @@ pafu_status pafu_workspace_status(const void* ws, void* stream);
 pafu_status pafu_score(const pafu_head* head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
                        float* scores, void* ws, size_t ws_bytes, void* stream);
 
+/* Step 1 on the input the paper feeds its head (Sec. 3.3 "Salience Estimation Head"; Appendix A
+ * "S-MLP": 4608 = 3 x 1536 inputs, 1024 hidden, 12 outputs, SiLU, mean over the outputs): token
+ * t's feature vector is the concatenation [q_t, k_t, v_t] of its query, key and value rows.
+ * The three matrices are read in place (no concatenated copy is made); everything else is as
+ * pafu_score with x_t = [q_t, k_t, v_t], so W1's columns are ordered query, key, value.
+ *   Q, K, V   device bf16 [n_tokens, ld] each, head->d_in / 3 features per row, ld % 8 == 0
+ * Supported: head->d_in % 192 == 0 (each third a multiple of 64), else as pafu_score. */
+pafu_status pafu_score_qkv(const pafu_head* head, const uint16_t* Q, const uint16_t* K, const uint16_t* V,
+                           int64_t n_tokens, int64_t ld, float* scores, void* ws, size_t ws_bytes, void* stream);
+
 /* Step 2 - retained indices (Sec. 3.4 inference paragraph; Algorithm 2 "Top-k"; frame sink
  * Sec. 4.1).  Per stream with T tokens and (n_sink, n_recent, budget):
  *   T <= budget            : keep all T tokens;

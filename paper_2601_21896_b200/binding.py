@@ -27,7 +27,7 @@ STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET
                 8: "PAFU_ERR_TOO_LARGE"}
 
 EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
-           "pafu_workspace_status", "pafu_score", "pafu_select", "pafu_compact",
+           "pafu_workspace_status", "pafu_score", "pafu_score_qkv", "pafu_select", "pafu_compact",
            "pafu_chunk_attn", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host"]
 
 
@@ -96,6 +96,8 @@ def lib() -> ctypes.CDLL:
         L.pafu_workspace_status.argtypes = [vp, vp]
         L.pafu_score.restype = i32
         L.pafu_score.argtypes = [ctypes.POINTER(CHead), vp, i64, i64, vp, vp, sz, vp]
+        L.pafu_score_qkv.restype = i32
+        L.pafu_score_qkv.argtypes = [ctypes.POINTER(CHead), vp, vp, vp, i64, i64, vp, vp, sz, vp]
         L.pafu_select.restype = i32
         L.pafu_select.argtypes = [vp, ctypes.POINTER(CShape), ctypes.POINTER(CPolicy), vp, vp, sz, vp]
         L.pafu_compact.restype = i32
@@ -206,6 +208,16 @@ def pafu_score(head: Head, X: torch.Tensor, scores: torch.Tensor, ws: Optional[t
     _check(lib().pafu_score(ctypes.byref(head.c), _ptr(X), n, ld, _ptr(scores), _ptr(ws),
                             0 if ws is None else ws.numel() * ws.element_size(), _stream()),
            "pafu_score")
+
+
+def pafu_score_qkv(head: Head, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, scores: torch.Tensor,
+                   ws: Optional[torch.Tensor] = None, n_tokens: Optional[int] = None,
+                   ld: Optional[int] = None) -> None:
+    n = K.shape[0] if n_tokens is None else n_tokens
+    stride = (K.numel() // max(K.shape[0], 1)) if ld is None else ld
+    _check(lib().pafu_score_qkv(ctypes.byref(head.c), _ptr(Q), _ptr(K), _ptr(V), n, stride, _ptr(scores), _ptr(ws),
+                                0 if ws is None else ws.numel() * ws.element_size(), _stream()),
+           "pafu_score_qkv")
 
 
 def pafu_select(scores: torch.Tensor, shape: Shape, policy, idx: torch.Tensor,

@@ -132,20 +132,40 @@ pafu_status pafu_workspace_status(const void* ws, void* stream) {
     return word == 0 ? PAFU_OK : PAFU_ERR_TIMEOUT;
 }
 
-pafu_status pafu_score(const pafu_head* head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
+namespace {
+// shared by the one- and three-matrix entry points; X[i] holds features [i * d_in / n_parts, ...)
+pafu_status score_impl(const pafu_head* head, const uint16_t* const* X, int n_parts, int64_t n_tokens, int64_t ldx,
                        float* scores, void* ws, size_t ws_bytes, void* stream) {
     pafu_status e = head_ok(head);
     if (e != PAFU_OK) return e;
+    if (head->d_in % (64 * n_parts) != 0) return PAFU_ERR_UNSUPPORTED_SHAPE;
     if (n_tokens < 0) return PAFU_ERR_INVALID_ARG;
     if (n_tokens == 0) return PAFU_OK;
-    if (X == nullptr || scores == nullptr) return PAFU_ERR_INVALID_ARG;
-    if (ldx < head->d_in || ldx % 8 != 0) return PAFU_ERR_INVALID_ARG;
-    if (!aligned16(X) || !aligned16(scores)) return PAFU_ERR_MISALIGNED;
+    if (scores == nullptr) return PAFU_ERR_INVALID_ARG;
+    for (int i = 0; i < n_parts; ++i)
+        if (X[i] == nullptr) return PAFU_ERR_INVALID_ARG;
+    if (ldx < head->d_in / n_parts || ldx % 8 != 0) return PAFU_ERR_INVALID_ARG;
+    for (int i = 0; i < n_parts; ++i)
+        if (!aligned16(X[i])) return PAFU_ERR_MISALIGNED;
+    if (!aligned16(scores)) return PAFU_ERR_MISALIGNED;
     const size_t need = kWsHeaderBytes + score_workspace_bytes(*head);
     if (ws == nullptr) return PAFU_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
     if (ws_bytes < need) return PAFU_ERR_WORKSPACE_TOO_SMALL;
-    return launch_score(*head, X, n_tokens, ldx, scores, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+    return launch_score(*head, X, n_parts, n_tokens, ldx, scores, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+}  // namespace
+
+pafu_status pafu_score(const pafu_head* head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
+                       float* scores, void* ws, size_t ws_bytes, void* stream) {
+    const uint16_t* parts[1] = {X};
+    return score_impl(head, parts, 1, n_tokens, ldx, scores, ws, ws_bytes, stream);
+}
+
+pafu_status pafu_score_qkv(const pafu_head* head, const uint16_t* Q, const uint16_t* K, const uint16_t* V,
+                           int64_t n_tokens, int64_t ld, float* scores, void* ws, size_t ws_bytes, void* stream) {
+    const uint16_t* parts[3] = {Q, K, V};
+    return score_impl(head, parts, 3, n_tokens, ld, scores, ws, ws_bytes, stream);
 }
 
 pafu_status pafu_select(const float* scores, const pafu_shape* shape, const pafu_policy* policy,

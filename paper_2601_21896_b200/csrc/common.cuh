@@ -76,7 +76,7 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 }
 
 // Launchers (each enqueues on `stream` and returns the launch status).
-pafu_status launch_score(const pafu_head& head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
+pafu_status launch_score(const pafu_head& head, const uint16_t* const* X, int n_parts, int64_t n_tokens, int64_t ldx,
                          float* scores, void* ws, size_t ws_bytes, cudaStream_t stream);
 pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* idx,
                           cudaStream_t stream);

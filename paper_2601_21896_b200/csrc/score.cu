@@ -6,10 +6,10 @@ namespace pafu {
 
 size_t score_workspace_bytes(const pafu_head&) { return 0; }
 
-pafu_status launch_score(const pafu_head& head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
+pafu_status launch_score(const pafu_head& head, const uint16_t* const* X, int n_parts, int64_t n_tokens, int64_t ldx,
                          float* scores, void* ws, size_t, cudaStream_t stream) {
     if (n_tokens == 0) return PAFU_OK;
-    return score_tc::launch(head, X, n_tokens, ldx, scores,
+    return score_tc::launch(head, X, n_parts, n_tokens, ldx, scores,
                             reinterpret_cast<int*>(ws) + kStatusWordTimeout, device_sm_count(), stream);
 }
 

@@ -14,8 +14,14 @@
 //   warp  9    TMA loader, 4-stage ring of {X 128x64, W1 256x64} tiles
 // Hidden units are processed in chunks of up to 256 (one accumulator of 256 TMEM columns);
 // two accumulators alternate so the read-out of one chunk overlaps the MMAs of the next.
+// When the token tiles alone would leave SMs idle (few tokens, a wide head) the kernel is
+// launched in clusters of n_chunks CTAs instead: each CTA takes one 256-unit chunk of one tile,
+// the partial row sums meet in the first CTA's shared memory (distributed shared memory) and are
+// added there in chunk order, so the result does not depend on timing.
 // All mbarrier waits are bounded (see sm100.cuh).
 #pragma once
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -33,11 +39,14 @@ constexpr int kXBytes = kBM * kBK * 2;          // 16 KiB
 constexpr int kWBytes = kNMax * kBK * 2;        // 32 KiB
 constexpr int kStageBytes = kXBytes + kWBytes;
 constexpr int kMaxHidden = 1024;
-constexpr int kSmemBytes = kStages * kStageBytes + 2 * kMaxHidden * 4 + 2 * kBM * 4 + 256 + 1024;
+constexpr int kMaxChunks = kMaxHidden / kNMax;
+constexpr int kSmemBytes = kStages * kStageBytes + 2 * kMaxHidden * 4 + 2 * kBM * 4 + kMaxChunks * kBM * 4 + 256 + 1024;
 
 struct Params {
     int64_t n_tokens;
     int d_in, d_hidden, d_out, act, final;
+    int k_per_part;      // reduction slices (of kBK features) taken from each input matrix
+    int split;           // 1: one (tile, chunk) per CTA, clusters of n_chunks CTAs
     const uint16_t* w2;
     const uint16_t* b1;
     const uint16_t* b2;
@@ -71,7 +80,8 @@ __device__ __forceinline__ float act_fn(float x) { return ACT == PAFU_ACT_GELU ?
 
 template <int ACT>
 __global__ void __launch_bounds__(kThreads, 1)
-score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ CUtensorMap mW,
+score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ CUtensorMap mX1,
+                const __grid_constant__ CUtensorMap mX2, const __grid_constant__ CUtensorMap mW,
                 const __grid_constant__ Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -79,7 +89,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
     float* w2m = reinterpret_cast<float*>(smem + kStages * kStageBytes);
     float* b1s = w2m + kMaxHidden;
     float* half_sum = b1s + kMaxHidden;                      // [2][kBM]: partial of column-half 1
-    uint64_t* bars = reinterpret_cast<uint64_t*>(half_sum + 2 * kBM);
+    float* chunk_sum = half_sum + 2 * kBM;                   // [kMaxChunks][kBM]: per-chunk row sums (split mode, first CTA)
+    uint64_t* bars = reinterpret_cast<uint64_t*>(chunk_sum + kMaxChunks * kBM);
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int st) { return bar0 + 8 * st; };
     auto empty = [&](int st) { return bar0 + 8 * (kStages + st); };
@@ -93,6 +104,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
     const int64_t n_tiles = (p.n_tokens + kBM - 1) / kBM;
     const int n_chunks = (p.d_hidden + kNMax - 1) / kNMax;
     const int n_k = p.d_in / kBK;
+    // work of this CTA: tiles tile0, tile0 + tile_step, ... and chunks [ch0, ch1) of each
+    const int64_t tile0 = p.split ? blockIdx.x / n_chunks : blockIdx.x;
+    const int64_t tile_step = p.split ? n_tiles : gridDim.x;
+    const int ch0 = p.split ? (int)(blockIdx.x % n_chunks) : 0;
+    const int ch1 = p.split ? ch0 + 1 : n_chunks;
 
     if (tid == 0) {
         for (int st = 0; st < kStages; ++st) { mbar_init(full(st), 1); mbar_init(empty(st), 1); }
@@ -129,16 +145,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
         // ---------------------------------------------------------------------- TMA loader
         if (elect_one()) {
             prefetch_tmap(&mX); prefetch_tmap(&mW);
+            if (p.k_per_part < n_k) { prefetch_tmap(&mX1); prefetch_tmap(&mX2); }
             uint32_t ring = 0;
             bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                for (int ch = 0; ch < n_chunks && ok; ++ch) {
+            for (int64_t tile = tile0; tile < n_tiles && ok; tile += tile_step) {
+                for (int ch = ch0; ch < ch1 && ok; ++ch) {
                     for (int k = 0; k < n_k; ++k, ++ring) {
                         const int st = ring % kStages;
                         if (abort_flag || !mbar_wait(empty(st), ((ring / kStages) & 1u) ^ 1u)) { fail(401); ok = false; break; }
                         const uint32_t dst = sStage + st * kStageBytes;
                         mbar_arrive_expect_tx(full(st), kStageBytes);
-                        tma_load_2d(dst, &mX, full(st), k * kBK, (int)(tile * kBM));
+                        // a token's features are the concatenation of its rows in up to three matrices
+                        const int part = k / p.k_per_part;
+                        const CUtensorMap* mx = part == 0 ? &mX : (part == 1 ? &mX1 : &mX2);
+                        tma_load_2d(dst, mx, full(st), (k - part * p.k_per_part) * kBK, (int)(tile * kBM));
                         tma_load_2d(dst + kXBytes, &mW, full(st), k * kBK, ch * kNMax);
                     }
                 }
@@ -154,8 +174,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
             const uint64_t desc0 = make_smem_desc_sw128(0, 16, 1024);
             uint32_t ring = 0, acc_it = 0;
             bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                for (int ch = 0; ch < n_chunks && ok; ++ch, ++acc_it) {
+            for (int64_t tile = tile0; tile < n_tiles && ok; tile += tile_step) {
+                for (int ch = ch0; ch < ch1 && ok; ++ch, ++acc_it) {
                     const int buf = acc_it & 1;
                     const int nc = min(kNMax, p.d_hidden - ch * kNMax);
                     const uint32_t idesc = make_idesc_bf16(kBM, nc, false, false);
@@ -184,9 +204,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
         const int row = quad * 32 + lane;
         uint32_t acc_it = 0, tile_it = 0;
         bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
+        for (int64_t tile = tile0; tile < n_tiles && ok; tile += tile_step, ++tile_it) {
             float part = 0.f;
-            for (int ch = 0; ch < n_chunks; ++ch, ++acc_it) {
+            for (int ch = ch0; ch < ch1; ++ch, ++acc_it) {
                 const int buf = acc_it & 1;
                 const int nc = min(kNMax, p.d_hidden - ch * kNMax);
                 {
@@ -219,11 +239,28 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
                 const bool w = mbar_wait(halves_bar, tile_it & 1u) && !abort_flag;
                 if (!__all_sync(0xffffffffu, w)) { fail(405); ok = false; break; }
                 const int64_t t = tile * kBM + row;
-                if (t < p.n_tokens) {
+                if (p.split) {
+                    // this chunk's row sums go to the cluster's first CTA
+                    cooperative_groups::this_cluster().map_shared_rank(chunk_sum, 0)[ch0 * kBM + row] = part + hs[row];
+                } else if (t < p.n_tokens) {
                     float v = part + hs[row] + b2m;
                     if (p.final == PAFU_FINAL_SIGMOID) v = rcpf(1.0f + ex2f(-v * 1.4426950408889634f));
                     p.scores[t] = v;
                 }
+            }
+        }
+    }
+    if (p.split) {
+        // every thread of the cluster gets here (all loops above are bounded)
+        cooperative_groups::this_cluster().sync();
+        if (ch0 == 0 && tid < kBM) {
+            const int64_t t = tile0 * kBM + tid;
+            if (t < p.n_tokens) {
+                float v = chunk_sum[tid];
+                for (int c = 1; c < n_chunks; ++c) v += chunk_sum[c * kBM + tid];
+                v += b2m;
+                if (p.final == PAFU_FINAL_SIGMOID) v = rcpf(1.0f + ex2f(-v * 1.4426950408889634f));
+                p.scores[t] = v;
             }
         }
     }
@@ -232,18 +269,28 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
     if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
-inline pafu_status launch(const pafu_head& head, const uint16_t* X, int64_t n_tokens, int64_t ldx,
+// X[0..n_parts) are the matrices whose rows, side by side, form a token's d_in features
+// (n_parts = 1: a plain [n_tokens, d_in] matrix; 3: query, key and value rows of d_in / 3 each).
+inline pafu_status launch(const pafu_head& head, const uint16_t* const* X, int n_parts, int64_t n_tokens, int64_t ldx,
                           float* scores, int* status, int sm_count, cudaStream_t stream) {
-    CUtensorMap mX, mW;
-    if (!TmapEncoder::matrix(&mX, X, (uint64_t)n_tokens, (uint64_t)head.d_in, (uint64_t)ldx, kBM)) return PAFU_ERR_CUDA;
+    CUtensorMap mX[3], mW;
+    const int d_part = head.d_in / n_parts;
+    for (int i = 0; i < 3; ++i)
+        if (!TmapEncoder::matrix(&mX[i], X[i < n_parts ? i : 0], (uint64_t)n_tokens, (uint64_t)d_part, (uint64_t)ldx, kBM))
+            return PAFU_ERR_CUDA;
     if (!TmapEncoder::matrix(&mW, head.w1, (uint64_t)head.d_hidden, (uint64_t)head.d_in, (uint64_t)head.d_in, kNMax))
         return PAFU_ERR_CUDA;
     Params p;
     p.n_tokens = n_tokens; p.d_in = head.d_in; p.d_hidden = head.d_hidden; p.d_out = head.d_out;
     p.act = head.act; p.final = head.final; p.w2 = head.w2; p.b1 = head.b1; p.b2 = head.b2;
     p.scores = scores; p.status = status;
+    p.k_per_part = d_part / kBK;
     const int64_t n_tiles = (n_tokens + kBM - 1) / kBM;
-    const int grid = (int)(n_tiles < sm_count ? n_tiles : sm_count);
+    const int n_chunks = (head.d_hidden + kNMax - 1) / kNMax;
+    // few tokens and a wide head: one CTA per (tile, chunk), clusters of n_chunks CTAs
+    p.split = (n_chunks > 1 && n_tiles * n_chunks <= 2 * (int64_t)sm_count) ? 1 : 0;
+    const int grid = p.split ? (int)(n_tiles * n_chunks) : (int)(n_tiles < sm_count ? n_tiles : sm_count);
+    const unsigned cluster = p.split ? (unsigned)n_chunks : 1u;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(score_tc_kernel<PAFU_ACT_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
@@ -252,8 +299,8 @@ inline pafu_status launch(const pafu_head& head, const uint16_t* X, int64_t n_to
         attr_set = true;
     }
     return cuda_ok(head.act == PAFU_ACT_GELU
-                       ? launch_dependent(score_tc_kernel<PAFU_ACT_GELU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mX, mW, p)
-                       : launch_dependent(score_tc_kernel<PAFU_ACT_SILU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mX, mW, p));
+                       ? launch_dependent(score_tc_kernel<PAFU_ACT_GELU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, cluster, mX[0], mX[1], mX[2], mW, p)
+                       : launch_dependent(score_tc_kernel<PAFU_ACT_SILU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, cluster, mX[0], mX[1], mX[2], mW, p));
 }
 
 }  // namespace score_tc

@@ -72,6 +72,12 @@ def test_argument_errors_are_caught_on_the_host(L):
     assert L.pafu_score(ctypes.byref(bad), fake, 4, 128, fake, None, 0, None) == 3
     bad = B.CHead(128, 32, 1, 7, 0, fake, None, fake, None)
     assert L.pafu_score(ctypes.byref(bad), fake, 4, 128, fake, None, 0, None) == 1
+    qkv = B.CHead(384, 32, 1, 0, 0, fake, None, fake, None)
+    assert L.pafu_score_qkv(ctypes.byref(qkv), fake, fake, None, 4, 128, fake, None, 0, None) == 1      # V missing
+    assert L.pafu_score_qkv(ctypes.byref(qkv), fake, fake, fake, 4, 64, fake, None, 0, None) == 1        # ld < d_in / 3
+    assert L.pafu_score_qkv(ctypes.byref(qkv), fake, fake + 2, fake, 4, 128, fake, None, 0, None) == 5  # misaligned K
+    assert L.pafu_score_qkv(ctypes.byref(head), fake, fake, fake, 4, 128, fake, None, 0, None) == 3      # 128 is not 3 x 64 k
+    assert L.pafu_score_qkv(ctypes.byref(qkv), fake, fake, fake, 0, 128, fake, None, 0, None) == 0      # empty: no-op
     assert L.pafu_select(None, ctypes.byref(sh.c), pol, fake, None, 0, None) == 1
     assert L.pafu_select(fake, ctypes.byref(sh.c), None, fake, None, 0, None) == 1
     assert L.pafu_select(fake, ctypes.byref(sh.c), pafu.make_policy(-1, 0, 5, 1), fake, None, 0, None) == 2

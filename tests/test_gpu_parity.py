@@ -87,6 +87,37 @@ def test_score_head_variants(act, final, d_out, d_hidden, n):
         close(out.cpu().numpy(), want, "score variant")
 
 
+@pytest.mark.parametrize("d_part,d_hidden,d_out,act,n,ld_extra", [
+    (1536, 1024, 12, wl.ACT_SILU, 4680, 0),    # the paper's S-MLP on one 3-frame chunk (Sec. 3.3, Appendix A)
+    (128, 64, 1, wl.ACT_GELU, 301, 64),        # rows wider than the features used, ragged last tile
+    (64, 272, 3, wl.ACT_SILU, 1, 0),
+])
+def test_score_qkv_matches_oracle_on_concatenated_rows(d_part, d_hidden, d_out, act, n, ld_extra):
+    """x_t = [q_t, k_t, v_t] read from three matrices in place equals the plain head applied to
+    the concatenated rows (the oracle sees only the concatenation)."""
+    rng = np.random.default_rng(11)
+    d_in = 3 * d_part
+    ld = d_part + ld_extra
+    bits = lambda shape, s=1.0: wl.f32_to_bf16_bits((rng.standard_normal(shape) * s).astype(np.float32))
+    Q, K, V = bits((n, ld)), bits((n, ld)), bits((n, ld))
+    w1 = bits((d_hidden, d_in), d_in ** -0.5); b1 = bits((d_hidden,), 0.3)
+    w2 = bits((d_out, d_hidden), d_hidden ** -0.5); b2 = bits((d_out,), 0.3)
+    dev = [to_device_bf16(a) for a in (Q, K, V, w1, b1, w2, b2)]
+    head = pafu.Head(dev[3], dev[4], dev[5], dev[6], act, wl.FINAL_NONE)
+    shape = pafu.Shape(3, 128, [0, n], [0, 1])
+    ws = torch.zeros(pafu.pafu_workspace_bytes(shape, None, head), dtype=torch.uint8, device="cuda")
+    out = torch.full((n,), float("nan"), device="cuda")
+    pafu.pafu_score_qkv(head, dev[0], dev[1], dev[2], out, ws, ld=ld)
+    assert pafu.pafu_workspace_status(ws) == 0
+    X = np.ascontiguousarray(np.concatenate([Q[:, :d_part], K[:, :d_part], V[:, :d_part]], axis=1))
+    want = oracle.score(X, w1, b1, w2, b2, act, wl.FINAL_NONE)
+    close(out.cpu().numpy(), want, "score qkv")
+    # and the one-matrix entry on the same concatenation gives the same bits
+    out1 = torch.full((n,), float("nan"), device="cuda")
+    pafu.pafu_score(head, to_device_bf16(X), out1, ws)
+    assert torch.equal(out, out1)
+
+
 # -------------------------------------------------------------------------------- select
 @pytest.mark.parametrize("kind", ["normal", "ties", "equal", "saturated", "heavy", "signed_zero"])
 def test_select_bit_exact(kind):
