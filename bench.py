@@ -313,6 +313,34 @@ def run_ours(args):
     ms_per_step = total_ms / steps
     value = world * n_layers * work["attn_flops"] / (ms_per_step * 1e-3) / 1e12
 
+    # ---- the same step with Select(KV; ids) applied inside the attention loader (no compaction
+    # copy): whole steps, then the indexed attention alone on the indices the steps left behind
+    indexed = None
+    if w.d_head == 128:
+        for i in range(3 * n_layers):
+            layers[i % n_sets].step_indexed()
+        i0, i1 = new_events(2)
+        torch.cuda.synchronize()
+        i0.record(stream)
+        for i in range(steps * n_layers):
+            layers[i % n_sets].step_indexed()
+        i1.record(stream)
+        torch.cuda.synchronize()
+        idx_ms = sharding.max_over_ranks(i0.elapsed_time(i1) / steps, device="cuda")
+        ev_a = [new_events(2) for _ in range(min(steps, 50))]
+        for i, (a, b) in enumerate(ev_a):
+            a.record(stream)
+            layers[i % n_sets].attn_indexed()
+            b.record(stream)
+        torch.cuda.synchronize()
+        for L in layers:
+            L.check_status()
+        ia_ms = float(np.mean([a.elapsed_time(b) for a, b in ev_a]))
+        indexed = {"api": "pafu_step_indexed (score, select, attention reading K/V rows through idx)",
+                   "ms_per_step": idx_ms,
+                   "value": world * n_layers * work["attn_flops"] / (idx_ms * 1e-3) / 1e12, "unit": UNIT,
+                   "attn_ms": ia_ms, "attn_TFLOP/s": work["attn_flops"] / (ia_ms * 1e-3) / 1e12}
+
     # ---- e2e: host buffers through pafu_step_host (H2D of inputs + D2H of results timed)
     L0 = layers[0]
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
@@ -411,6 +439,7 @@ def run_ours(args):
                                 k_ms[:3].sum()) / peaks["hbm_gbs"]},
         },
         "score_qkv": qkv,
+        "step_indexed": indexed,
         "layers_per_step": n_layers,
         "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step / n_layers,
         "peaks": peaks,

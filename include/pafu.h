@@ -187,6 +187,23 @@ pafu_status pafu_chunk_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_
                             const pafu_shape* shape, float scale, uint16_t* O, float* LSE,
                             void* ws, size_t ws_bytes, void* stream);
 
+/* Step 4 without step 3 - chunk attention that reads the retained tokens through the index list
+ * ("index-based cache management": Sec. 3.4, Eq. 7 restricts attention to the index set I_s of the
+ * full cache instead of to a copied cache).  Computes exactly what pafu_compact followed by
+ * pafu_chunk_attn computes - the outputs are bit-identical - but K and V are the UNCOMPACTED
+ * cache and the loader fetches rows idx[.] of it, so no compacted copy is written or read.
+ *   K, V      device bf16 [cu_T[n_streams], n_heads, d_head], the cache before pruning
+ *   idx       device int32 [cu_B[n_streams]] as written by pafu_select: per stream, stream-local
+ *             token indices in [0, T_s), at offset cu_B[s]
+ *   cu_B      HOST prefix array of retained tokens (pafu_kept_counts); B_s <= T_s
+ *   shape     needs both cu_T and cu_Lq
+ * Everything else as pafu_chunk_attn.  Supported: d_head = 128; every stream with queries needs
+ * at least one key; total cache rows < 2^31. */
+pafu_status pafu_chunk_attn_indexed(const uint16_t* Q, const uint16_t* K, const uint16_t* V, const int32_t* idx,
+                                    const int64_t* cu_B, const uint16_t* Kq, const uint16_t* Vq,
+                                    const pafu_shape* shape, float scale, uint16_t* O, float* LSE,
+                                    void* ws, size_t ws_bytes, void* stream);
+
 /* Chunk attention without a workspace - the paper has no counterpart; this entry point exists
  * for callers that are not allowed to allocate device memory: code running inside another
  * framework's memory plan or a fixed-memory service, plug-ins handed only their input and
@@ -240,6 +257,12 @@ typedef struct pafu_step_args {
  * pafu_select, pafu_compact and pafu_chunk_attn produce when called in sequence with the
  * same buffers (the salience head reads each token's K across all heads). */
 pafu_status pafu_step(const pafu_step_args* args, void* stream);
+
+/* The layer step without the compaction copy: score, Top-k, then pafu_chunk_attn_indexed on the
+ * uncompacted cache (Algorithm 2 with Select(KV; ids) applied inside the attention's loader).
+ * args->Kc, Vc, SLc are ignored (may be NULL); scores, idx, O (and LSE) are written and equal
+ * pafu_step's bit for bit.  d_head = 128 only. */
+pafu_status pafu_step_indexed(const pafu_step_args* args, void* stream);
 
 /* pafu_step with timestamps: identical launches, plus five caller-created CUDA events
  * (HOST array of 5 cudaEvent_t passed as void*) recorded on `stream` before the score step and

@@ -28,7 +28,7 @@ STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET
 
 EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
            "pafu_workspace_status", "pafu_score", "pafu_score_qkv", "pafu_select", "pafu_compact",
-           "pafu_chunk_attn", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host"]
+           "pafu_chunk_attn", "pafu_chunk_attn_indexed", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_indexed", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host"]
 
 
 class PafuError(RuntimeError):
@@ -106,6 +106,11 @@ def lib() -> ctypes.CDLL:
         L.pafu_chunk_attn.restype = i32
         L.pafu_chunk_attn.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.POINTER(CShape),
                                       ctypes.c_float, vp, vp, vp, sz, vp]
+        L.pafu_chunk_attn_indexed.restype = i32
+        L.pafu_chunk_attn_indexed.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(CShape),
+                                              ctypes.c_float, vp, vp, vp, sz, vp]
+        L.pafu_step_indexed.restype = i32
+        L.pafu_step_indexed.argtypes = [ctypes.POINTER(CStepArgs), vp]
         L.pafu_chunk_attn_noalloc.restype = i32
         L.pafu_chunk_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.POINTER(CShape),
                                               ctypes.c_float, vp, vp, vp]
@@ -241,6 +246,16 @@ def pafu_chunk_attn(Q, Kc, Vc, cu_B, Kq, Vq, shape: Shape, scale: float, O, LSE=
            "pafu_chunk_attn")
 
 
+def pafu_chunk_attn_indexed(Q, K, V, idx, cu_B, Kq, Vq, shape: Shape, scale: float, O, LSE=None,
+                            ws: Optional[torch.Tensor] = None) -> None:
+    """Chunk attention over rows idx[.] of the uncompacted cache K, V (no compacted copy)."""
+    cu_B = np.ascontiguousarray(cu_B, dtype=np.int64)
+    _check(lib().pafu_chunk_attn_indexed(_ptr(Q), _ptr(K), _ptr(V), _ptr(idx), _ptr(cu_B), _ptr(Kq), _ptr(Vq),
+                                         ctypes.byref(shape.c), float(scale), _ptr(O), _ptr(LSE), _ptr(ws),
+                                         0 if ws is None else ws.numel() * ws.element_size(), _stream()),
+           "pafu_chunk_attn_indexed")
+
+
 def pafu_chunk_attn_noalloc(Q, Kc, Vc, cu_B, Kq, Vq, shape: Shape, scale: float, O, LSE=None) -> None:
     """Chunk attention that takes no workspace: its scratch is a fixed array inside the library
     (see include/pafu.h for the size limit and the rule that calls must not overlap)."""
@@ -262,6 +277,10 @@ def step_args(shape: Shape, head: Head, policy, K, V, Q, Kq, Vq, scale, scores, 
 
 def pafu_step(args: CStepArgs) -> None:
     _check(lib().pafu_step(ctypes.byref(args), _stream()), "pafu_step")
+
+
+def pafu_step_indexed(args: CStepArgs) -> None:
+    _check(lib().pafu_step_indexed(ctypes.byref(args), _stream()), "pafu_step_indexed")
 
 
 def event_handles(events: Sequence["torch.cuda.Event"]):

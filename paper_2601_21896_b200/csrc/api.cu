@@ -235,6 +235,44 @@ pafu_status pafu_chunk_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_
                        static_cast<cudaStream_t>(stream));
 }
 
+pafu_status pafu_chunk_attn_indexed(const uint16_t* Q, const uint16_t* K, const uint16_t* V, const int32_t* idx,
+                                    const int64_t* cu_B, const uint16_t* Kq, const uint16_t* Vq,
+                                    const pafu_shape* shape, float scale, uint16_t* O, float* LSE,
+                                    void* ws, size_t ws_bytes, void* stream) {
+    pafu_status e = shape_ok(shape, true, true);
+    if (e != PAFU_OK) return e;
+    if (shape->d_head != 128) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    if (!prefix_ok(cu_B, shape->n_streams)) return PAFU_ERR_INVALID_ARG;
+    if (!(scale >= 0.f) || isinf(scale)) return PAFU_ERR_INVALID_ARG;
+    StreamTable st;
+    memset(&st, 0, sizeof st);
+    st.n_streams = shape->n_streams;
+    fill_prefix(st.cu_T, shape->cu_T, shape->n_streams);
+    fill_prefix(st.cu_Lq, shape->cu_Lq, shape->n_streams);
+    fill_prefix(st.cu_B, cu_B, shape->n_streams);
+    for (int s = 0; s < st.n_streams; ++s) {
+        if (st.cu_B[s + 1] - st.cu_B[s] > st.cu_T[s + 1] - st.cu_T[s]) return PAFU_ERR_INVALID_ARG;
+    }
+    if (st.cu_T[st.n_streams] > 0x7fffffffLL) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    if (st.cu_Lq[st.n_streams] == 0) return PAFU_OK;
+    if (Q == nullptr || O == nullptr) return PAFU_ERR_INVALID_ARG;
+    if ((Kq == nullptr) != (Vq == nullptr)) return PAFU_ERR_INVALID_ARG;
+    if (st.cu_B[st.n_streams] > 0 && (K == nullptr || V == nullptr || idx == nullptr)) return PAFU_ERR_INVALID_ARG;
+    if (!aligned16(Q) || !aligned16(O) || !aligned16(K) || !aligned16(V) || !aligned16(Kq) ||
+        !aligned16(Vq) || !aligned16(LSE) || !aligned16(idx)) return PAFU_ERR_MISALIGNED;
+    if (!attn_indexed_supported(st, shape->d_head, Kq != nullptr)) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    const size_t need = kWsHeaderBytes + attn_workspace_bytes(st, shape->n_heads, shape->d_head);
+    if (ws == nullptr) return PAFU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
+    if (ws_bytes < need) return PAFU_ERR_WORKSPACE_TOO_SMALL;
+    if (scale == 0.f) scale = 1.0f / sqrtf((float)shape->d_head);
+    if (st.cu_B[st.n_streams] == 0)      // nothing retained: the plain kernel over the chunk's own tokens
+        return launch_attn(Q, nullptr, nullptr, Kq, Vq, st, shape->n_heads, shape->d_head, scale, O, LSE, ws, ws_bytes,
+                           static_cast<cudaStream_t>(stream));
+    return launch_attn_indexed(Q, K, V, idx, Kq, Vq, st, shape->n_heads, scale, O, LSE, ws, ws_bytes,
+                               static_cast<cudaStream_t>(stream));
+}
+
 static pafu_status step_impl(const pafu_step_args* a, void* const* ev, void* stream);
 
 pafu_status pafu_step(const pafu_step_args* a, void* stream) { return step_impl(a, nullptr, stream); }
@@ -244,6 +282,46 @@ pafu_status pafu_step_timed(const pafu_step_args* a, void* const* events, void* 
     for (int i = 0; i < 5; ++i)
         if (events[i] == nullptr) return PAFU_ERR_INVALID_ARG;
     return step_impl(a, events, stream);
+}
+
+pafu_status pafu_step_indexed(const pafu_step_args* a, void* stream) {
+    if (a == nullptr) return PAFU_ERR_INVALID_ARG;
+    pafu_status e = shape_ok(&a->shape, true, true);
+    if (e != PAFU_OK) return e;
+    e = head_ok(a->head);
+    if (e != PAFU_OK) return e;
+    const int64_t dm = (int64_t)a->shape.n_heads * a->shape.d_head;
+    if (a->head->d_in != dm) return PAFU_ERR_INVALID_ARG;
+    if (a->shape.d_head != 128) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    int64_t cu_B[PAFU_MAX_STREAMS + 1];
+    e = pafu_kept_counts(&a->shape, a->policy, cu_B);
+    if (e != PAFU_OK) return e;
+    const int n = a->shape.n_streams;
+    const int64_t nT = a->shape.cu_T[n], nB = cu_B[n], nQ = a->shape.cu_Lq[n];
+    if (nT > 0 && (a->K == nullptr || a->V == nullptr || a->scores == nullptr)) return PAFU_ERR_INVALID_ARG;
+    if (nB > 0 && a->idx == nullptr) return PAFU_ERR_INVALID_ARG;
+    if (nQ > 0 && (a->Q == nullptr || a->O == nullptr)) return PAFU_ERR_INVALID_ARG;
+    if ((a->Kq == nullptr) != (a->Vq == nullptr)) return PAFU_ERR_INVALID_ARG;
+    if (!(a->scale >= 0.f) || isinf(a->scale)) return PAFU_ERR_INVALID_ARG;
+    const void* ptrs[] = {a->K, a->V, a->Q, a->Kq, a->Vq, a->scores, a->idx, a->O, a->LSE};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return PAFU_ERR_MISALIGNED;
+    StreamTable st;
+    memset(&st, 0, sizeof st);
+    st.n_streams = n;
+    fill_prefix(st.cu_Lq, a->shape.cu_Lq, n);
+    fill_prefix(st.cu_B, cu_B, n);
+    if (!attn_indexed_supported(st, a->shape.d_head, a->Kq != nullptr)) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    const size_t need = pafu_workspace_bytes(&a->shape, a->policy, a->head);
+    if (a->ws == nullptr) return PAFU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(a->ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
+    if (a->ws_bytes < need) return PAFU_ERR_WORKSPACE_TOO_SMALL;
+    e = pafu_score(a->head, a->K, nT, dm, a->scores, a->ws, a->ws_bytes, stream);
+    if (e != PAFU_OK) return e;
+    e = pafu_select(a->scores, &a->shape, a->policy, a->idx, a->ws, a->ws_bytes, stream);
+    if (e != PAFU_OK) return e;
+    return pafu_chunk_attn_indexed(a->Q, a->K, a->V, a->idx, cu_B, a->Kq, a->Vq, &a->shape, a->scale, a->O, a->LSE,
+                                   a->ws, a->ws_bytes, stream);
 }
 
 static pafu_status step_impl(const pafu_step_args* a, void* const* ev, void* stream) {

@@ -25,6 +25,22 @@ pafu_status launch_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_t* V
     return attn_mma::launch(Q, Kc, Vc, Kq, Vq, st, n_heads, d_head, scale, O, LSE, stream);
 }
 
+// Retained keys/values read through the index list from the uncompacted cache (d_head 128).
+pafu_status launch_attn_indexed(const uint16_t* Q, const uint16_t* K, const uint16_t* V, const int32_t* idx,
+                                const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
+                                int32_t n_heads, float scale, uint16_t* O, float* LSE,
+                                void* ws, size_t, cudaStream_t stream) {
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    return attn_tc::launch(Q, K, V, Kq, Vq, st, n_heads, scale, O, LSE,
+                           reinterpret_cast<int*>(base) + kStatusWordTimeout,
+                           reinterpret_cast<float*>(base + kWsHeaderBytes), stream, 0, idx,
+                           st.cu_T[st.n_streams]);
+}
+
+bool attn_indexed_supported(const StreamTable& st, int32_t d_head, bool has_chunk) {
+    return d_head == attn_tc::kD && attn_tc::supports(st, has_chunk);
+}
+
 }  // namespace pafu
 
 // ---------------------------------------------------------------------------------------------

@@ -77,6 +77,7 @@ struct Params {
     float* LSE;
     int* status;        // workspace status word (device)
     float* pieces;      // [gridDim][2][kPieceFloats]
+    const int32_t* idx; // gather variant: retained token indices, stream-local, [cu_B[n_streams]]
     int64_t total_Lq;
     int64_t total_cost;
 };
@@ -196,6 +197,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
+// GATHER = false: the retained keys/values are the rows of a compacted cache (mKc, mVc are tiled
+// maps of it).  GATHER = true: they are rows idx[.] of the uncompacted cache, fetched by the
+// loader four rows at a time (mKc, mVc are two-dimensional [tokens, n_heads * d_head] maps with a
+// one-row box); everything downstream of the shared-memory ring is identical.
+template <bool GATHER>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mKc,
                const __grid_constant__ CUtensorMap mVc, const __grid_constant__ CUtensorMap mKq,
@@ -254,7 +260,79 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
         // idle
     } else if (warp == 9) {
         // ------------------------------------------------------------------ TMA loader
-        if (elect_one()) {
+        if constexpr (GATHER) {
+            // The whole warp walks the runs together.  Lane 0 issues the tiled loads (Q, the
+            // chunk's own K/V); a retained 64-key tile is 2 column halves x 16 groups of four
+            // rows, one gather per lane for K and one for V, each writing 4 x 128 bytes at the
+            // place the tiled load would have put those rows (the swizzle is a function of the
+            // shared-memory address, so the tile's layout is unchanged).
+            const int lane = tid & 31;
+            const int grp = lane & 15, half = lane >> 4;
+            if (lane == 0) {
+                prefetch_tmap(&mQ); prefetch_tmap(&mKc); prefetch_tmap(&mVc);
+                if (p.has_chunk) { prefetch_tmap(&mKq); prefetch_tmap(&mVq); }
+            }
+            SegIter iter(p, blockIdx.x, gridDim.x);
+            Seg g;
+            uint32_t ring = 0, qcnt0 = 0, qcnt1 = 0;
+            bool ok = true;
+            auto wait_all = [&](uint32_t bar, uint32_t ph, int code) {
+                const bool w = !abort_flag && mbar_wait(bar, ph);
+                if (!__all_sync(0xffffffffu, w)) { if (lane == 0) fail(code); ok = false; }
+            };
+            while (ok && iter.next(p, g)) {
+                const int qrow = (int)(p.st.cu_Lq[g.stream] + g.q0);
+                for (int s = 0; s < g.n_slots && ok; ++s) {
+                    const uint32_t qc = s ? qcnt1 : qcnt0;
+                    wait_all(q_empty(s), (qc & 1u) ^ 1u, 100);
+                    if (!ok) break;
+                    if (s) ++qcnt1; else ++qcnt0;
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(q_full(s), kQBytes);
+                        tma_load_3d(sQ + s * kQBytes, &mQ, q_full(s), 0, g.head, qrow + s * kBM);
+                        tma_load_3d(sQ + s * kQBytes + kQHalf, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
+                    }
+                }
+                const int32_t* sidx = p.idx + p.st.cu_B[g.stream];
+                const int row_base = (int)p.st.cu_T[g.stream];
+                for (int j = g.t0; j < g.t1 && ok; ++j) {
+                    const bool seg2 = j >= g.nt1;
+                    int r[4] = {0, 0, 0, 0};
+                    if (!seg2) {
+                        // rows past the segment's end repeat its last row: their logits are masked,
+                        // and their values must be finite
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            int64_t pos = (int64_t)j * kBN + grp * 4 + e;
+                            if (pos >= g.nB) pos = g.nB - 1;
+                            r[e] = row_base + __ldg(sidx + pos);
+                        }
+                    }
+                    const int row2 = (int)(p.st.cu_Lq[g.stream] + (int64_t)(j - g.nt1) * kBN);
+                    for (int kv = 0; kv < 2 && ok; ++kv, ++ring) {
+                        const int st = ring % kStages;
+                        wait_all(kv_empty(st), ((ring / kStages) & 1u) ^ 1u, 101);
+                        if (!ok) break;
+                        if (lane == 0) mbar_arrive_expect_tx(kv_full(st), kTileBytes);
+                        __syncwarp();
+                        if (seg2) {
+                            if (lane == 0) {
+                                const CUtensorMap* m = kv ? &mVq : &mKq;
+                                tma_load_3d(sKV + st * kTileBytes, m, kv_full(st), 0, g.head, row2);
+                                tma_load_3d(sKV + st * kTileBytes + kHalfBytes, m, kv_full(st), 64, g.head, row2);
+                            }
+                        } else {
+                            tma_gather4_2d(sKV + st * kTileBytes + half * kHalfBytes + grp * 512, kv ? &mVc : &mKc,
+                                           kv_full(st), g.head * kD + half * 64, r[0], r[1], r[2], r[3]);
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                for (uint32_t r = ring > (uint32_t)kStages ? ring - kStages : 0; r < ring; ++r)
+                    mbar_wait(kv_full(r % kStages), (r / kStages) & 1u);
+            }
+        } else if (elect_one()) {
             prefetch_tmap(&mQ); prefetch_tmap(&mKc); prefetch_tmap(&mVc);
             if (p.has_chunk) { prefetch_tmap(&mKq); prefetch_tmap(&mVq); }
             SegIter iter(p, blockIdx.x, gridDim.x);
@@ -693,7 +771,8 @@ inline size_t workspace_bytes() { return (size_t)sm_count() * 2 * kPieceBytes; }
 inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
                           const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
                           int32_t n_heads, float scale, uint16_t* O, float* LSE, int* status,
-                          float* pieces, cudaStream_t stream, int max_ctas = 0) {
+                          float* pieces, cudaStream_t stream, int max_ctas = 0,
+                          const int32_t* idx = nullptr, int64_t n_cache_rows = 0) {
     const int n = st.n_streams;
     const int64_t nQ = st.cu_Lq[n], nB = st.cu_B[n];
     const int has_chunk = Kq != nullptr;
@@ -701,7 +780,11 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
     if (cost == 0) return PAFU_OK;
     CUtensorMap mQ, mKc, mVc, mKq, mVq;
     if (!TmapEncoder::token_tensor(&mQ, Q, (uint64_t)nQ, n_heads, kD, kBM)) return PAFU_ERR_CUDA;
-    if (nB > 0) {
+    const bool gather = idx != nullptr;      // Kc, Vc are then the uncompacted cache of n_cache_rows tokens
+    if (nB > 0 && gather) {
+        if (!TmapEncoder::matrix(&mKc, Kc, (uint64_t)n_cache_rows, (uint64_t)n_heads * kD, (uint64_t)n_heads * kD, 1) ||
+            !TmapEncoder::matrix(&mVc, Vc, (uint64_t)n_cache_rows, (uint64_t)n_heads * kD, (uint64_t)n_heads * kD, 1)) return PAFU_ERR_CUDA;
+    } else if (nB > 0) {
         if (!TmapEncoder::token_tensor(&mKc, Kc, (uint64_t)nB, n_heads, kD, kBN) ||
             !TmapEncoder::token_tensor(&mVc, Vc, (uint64_t)nB, n_heads, kD, kBN)) return PAFU_ERR_CUDA;
     } else { mKc = mQ; mVc = mQ; }
@@ -711,16 +794,18 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
     } else { mKq = mQ; mVq = mQ; }
     Params p;
     p.st = st; p.n_heads = n_heads; p.has_chunk = has_chunk; p.scale = scale;
-    p.O = O; p.LSE = LSE; p.status = status; p.pieces = pieces; p.total_Lq = nQ; p.total_cost = cost;
+    p.O = O; p.LSE = LSE; p.status = status; p.pieces = pieces; p.idx = idx; p.total_Lq = nQ; p.total_cost = cost;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return PAFU_ERR_CUDA;
         attr_set = true;
     }
     int grid = grid_for(cost);
     if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;   // caller's scratch holds fewer partials
-    if (launch_dependent(attn_tc_kernel, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mKc, mVc, mKq, mVq, p) != cudaSuccess)
+    if ((gather ? launch_dependent(attn_tc_kernel<true>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mKc, mVc, mKq, mVq, p)
+                : launch_dependent(attn_tc_kernel<false>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mKc, mVc, mKq, mVq, p)) != cudaSuccess)
         return PAFU_ERR_CUDA;
     if (grid > 1) {
         if (launch_dependent(attn_tc_merge_kernel, dim3(2 * grid), dim3(1024), 0, stream, 1, p, grid) != cudaSuccess)

@@ -87,6 +87,11 @@ pafu_status launch_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_t* V
                         const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
                         int32_t n_heads, int32_t d_head, float scale, uint16_t* O, float* LSE,
                         void* ws, size_t ws_bytes, cudaStream_t stream);
+pafu_status launch_attn_indexed(const uint16_t* Q, const uint16_t* K, const uint16_t* V, const int32_t* idx,
+                                const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
+                                int32_t n_heads, float scale, uint16_t* O, float* LSE,
+                                void* ws, size_t ws_bytes, cudaStream_t stream);
+bool attn_indexed_supported(const StreamTable& st, int32_t d_head, bool has_chunk);
 size_t attn_workspace_bytes(const StreamTable& st, int32_t n_heads, int32_t d_head);
 size_t score_workspace_bytes(const pafu_head& head);
 

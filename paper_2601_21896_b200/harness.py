@@ -71,8 +71,15 @@ class Layer:
         B.pafu_chunk_attn(self.Q, self.Kc, self.Vc, self.cu_B, self.Kq, self.Vq, self.shape, 0.0,
                           self.O, self.LSE, self.ws)
 
+    def attn_indexed(self):
+        B.pafu_chunk_attn_indexed(self.Q, self.K, self.V, self.idx, self.cu_B, self.Kq, self.Vq,
+                                  self.shape, 0.0, self.O, self.LSE, self.ws)
+
     def step(self):
         B.pafu_step(self.args)
+
+    def step_indexed(self):
+        B.pafu_step_indexed(self.args)
 
     def check_status(self):
         st = B.pafu_workspace_status(self.ws)

@@ -219,6 +219,65 @@ def test_attention_segment_edge_cases():
             close(LSE.cpu().numpy(), wl_, "edge LSE")
 
 
+# --------------------------------------------------------------- attention through indices
+def test_indexed_attention_matches_oracle_and_compacted_path():
+    """Select(KV; ids) applied inside the attention loader (Eq. 7's index set) instead of as a
+    copy: against the oracle on the oracle's own gathered rows, and bit-equal to the CUDA path
+    that compacts first.  Retained counts sit around the 4-row gather and 64-key tile sizes;
+    streams have non-zero offsets into the packed cache."""
+    rng = np.random.default_rng(21)
+    N, D = 3, 128
+    for T, Bs, Lq, chunk in [((300,), (1,), (5,), False), ((300,), (3,), (70,), True),
+                             ((500, 129, 1000), (63, 129, 257), (130, 1, 300), True),
+                             ((257, 64), (65, 64), (256, 257), False),
+                             ((2000,), (1027,), (520,), True)]:
+        n = len(T)
+        cuT = np.concatenate([[0], np.cumsum(T)]); cuB = np.concatenate([[0], np.cumsum(Bs)])
+        cuQ = np.concatenate([[0], np.cumsum(Lq)])
+        bits = lambda m: wl.f32_to_bf16_bits(rng.standard_normal((m, N, D)).astype(np.float32))
+        K, V, Q, Kq, Vq = bits(cuT[-1]), bits(cuT[-1]), bits(cuQ[-1]), bits(cuQ[-1]), bits(cuQ[-1])
+        idx = np.concatenate([np.sort(rng.choice(T[s], size=Bs[s], replace=False)) for s in range(n)]).astype(np.int32)
+        shape = pafu.Shape(N, D, cuT, cuQ)
+        pol = pafu.make_policy(0, 0, list(Bs), n)
+        dK, dV, dQ, dKq, dVq = [to_device_bf16(a) for a in (K, V, Q, Kq, Vq)]
+        didx = torch.from_numpy(idx).cuda()
+        ws = torch.zeros(pafu.pafu_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+        O = torch.full((int(cuQ[-1]), N, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        LSE = torch.full((N, int(cuQ[-1])), float("nan"), device="cuda")
+        pafu.pafu_chunk_attn_indexed(dQ, dK, dV, didx, cuB, dKq if chunk else None, dVq if chunk else None,
+                                     shape, 0.0, O, LSE, ws)
+        assert pafu.pafu_workspace_status(ws) == 0
+        got = wl.bf16_bits_to_f32(bf16_to_bits(O)); lse = LSE.cpu().numpy()
+        for s in range(n):
+            i = idx[cuB[s]:cuB[s + 1]]
+            want, wlse = oracle.attention(Q[cuQ[s]:cuQ[s + 1]], oracle.compact(K[cuT[s]:cuT[s + 1]], i),
+                                          oracle.compact(V[cuT[s]:cuT[s + 1]], i),
+                                          Kq[cuQ[s]:cuQ[s + 1]] if chunk else None,
+                                          Vq[cuQ[s]:cuQ[s + 1]] if chunk else None)
+            close(got[cuQ[s]:cuQ[s + 1]], want, "indexed O %s stream %d" % ((T, Bs, Lq), s))
+            close(lse[:, cuQ[s]:cuQ[s + 1]], wlse, "indexed LSE")
+        # the compact-then-attend path on the same inputs gives the same bits
+        Kc = torch.zeros((int(cuB[-1]), N, D), dtype=torch.bfloat16, device="cuda"); Vc = torch.zeros_like(Kc)
+        pafu.pafu_compact(dK, dV, None, didx, shape, pol, Kc, Vc, None)
+        O2 = torch.full_like(O, float("nan")); LSE2 = torch.full_like(LSE, float("nan"))
+        pafu.pafu_chunk_attn(dQ, Kc, Vc, cuB, dKq if chunk else None, dVq if chunk else None, shape, 0.0, O2, LSE2, ws)
+        assert torch.equal(O.view(torch.int16), O2.view(torch.int16)) and torch.equal(LSE, LSE2)
+
+
+@pytest.mark.parametrize("w", [wl.small_ragged(2, 128), wl.wan13b_layer(), wl.batch4_14b()],
+                         ids=lambda w: w.name)
+def test_step_indexed_equals_step(w):
+    d = wl.make_layer(w)
+    A = Layer(w, d); B = Layer(w, d)
+    A.step(); A.check_status()
+    B.O.fill_(float("nan")); B.LSE.fill_(float("nan"))
+    B.step_indexed(); B.check_status()
+    assert torch.equal(A.scores[: A.nT], B.scores[: A.nT])
+    assert torch.equal(A.idx[: A.nB], B.idx[: A.nB])
+    assert torch.equal(A.O.view(torch.int16), B.O.view(torch.int16))
+    assert torch.equal(A.LSE, B.LSE)
+
+
 # ---------------------------------------------------------------------------------- step
 @pytest.mark.parametrize("w", SMALL, ids=lambda w: "%s-d%d" % (w.name, w.d_head))
 def test_step_equals_four_calls_and_oracle(w):
