@@ -284,6 +284,30 @@ size_t pafu_step_host_arena_bytes(const pafu_shape* shape, const pafu_policy* po
 pafu_status pafu_step_host(const pafu_step_args* args, void* arena, size_t arena_bytes,
                            void* stream);
 
+/* Teacher-side salience target - Spatialtemporal-balanced Salience Estimation (Sec. 3.2, Eq. 4
+ * and Eq. 5; Algorithm 3).  With P = softmax(scale * Q K^T) per head over the whole sequence of L
+ * tokens (bidirectional) and blocks of block_len tokens, key j gets
+ *   low_j  = mean over heads of max_i P[n,i,j] over the queries i of LATER blocks,
+ *   diag_j = the same over the queries of j's OWN block,
+ *   up_j   = the same over the queries of EARLIER blocks   (an empty set of queries gives 0),
+ * and s_j = (diag + low) / 2 for j < block_len, (up + diag + low) / 3 for
+ * block_len <= j < L - block_len, (diag + up) / 2 for the rest (the first matching case when
+ * L < 2 * block_len).  P is never written: the kernel needs only each row's log-sum-exp.
+ *   Q, K      device bf16 [L, n_heads, d_head]
+ *   LSE       device fp32 [n_heads, L]: log-sum-exp of scale * q_i . k_j over all L keys, as
+ *             pafu_chunk_attn writes it for the same Q, K and scale; NULL = computed here with the
+ *             attention kernel (costs a full attention pass and scratch for its output)
+ *   s         device fp32 [L], out
+ *   comp      device fp32 [3, L], out: low, diag, up; or NULL
+ *   ws        device workspace of pafu_sse_workspace_bytes(...), 256-byte aligned, status header
+ *             (first 256 bytes) zeroed by the caller; read it back with pafu_workspace_status
+ * Supported: d_head = 128, L < 2^31.  fp32 accumulation; results agree with the definition to
+ * about 1e-5 relative (the logits' rounding), not bit for bit. */
+size_t pafu_sse_workspace_bytes(int64_t L, int32_t n_heads, int32_t d_head, int64_t block_len);
+pafu_status pafu_sse(const uint16_t* Q, const uint16_t* K, const float* LSE, int64_t L,
+                     int32_t n_heads, int32_t d_head, int64_t block_len, float scale,
+                     float* s, float* comp, void* ws, size_t ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

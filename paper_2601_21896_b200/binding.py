@@ -28,7 +28,8 @@ STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET
 
 EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
            "pafu_workspace_status", "pafu_score", "pafu_score_qkv", "pafu_select", "pafu_compact",
-           "pafu_chunk_attn", "pafu_chunk_attn_indexed", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_indexed", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host"]
+           "pafu_chunk_attn", "pafu_chunk_attn_indexed", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_indexed", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host",
+           "pafu_sse_workspace_bytes", "pafu_sse"]
 
 
 class PafuError(RuntimeError):
@@ -111,6 +112,10 @@ def lib() -> ctypes.CDLL:
                                               ctypes.c_float, vp, vp, vp, sz, vp]
         L.pafu_step_indexed.restype = i32
         L.pafu_step_indexed.argtypes = [ctypes.POINTER(CStepArgs), vp]
+        L.pafu_sse_workspace_bytes.restype = sz
+        L.pafu_sse_workspace_bytes.argtypes = [i64, i32, i32, i64]
+        L.pafu_sse.restype = i32
+        L.pafu_sse.argtypes = [vp, vp, vp, i64, i32, i32, i64, ctypes.c_float, vp, vp, vp, sz, vp]
         L.pafu_chunk_attn_noalloc.restype = i32
         L.pafu_chunk_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.POINTER(CShape),
                                               ctypes.c_float, vp, vp, vp]
@@ -277,6 +282,17 @@ def step_args(shape: Shape, head: Head, policy, K, V, Q, Kq, Vq, scale, scores, 
 
 def pafu_step(args: CStepArgs) -> None:
     _check(lib().pafu_step(ctypes.byref(args), _stream()), "pafu_step")
+
+
+def pafu_sse_workspace_bytes(L: int, n_heads: int, d_head: int, block_len: int) -> int:
+    return lib().pafu_sse_workspace_bytes(L, n_heads, d_head, block_len)
+
+
+def pafu_sse(Q, K, LSE, block_len: int, scale: float, s, comp, ws) -> None:
+    """Teacher salience target (Eq. 4, Eq. 5) of Q, K [L, N, D]; LSE [N, L] or None."""
+    L, N, D = Q.shape
+    _check(lib().pafu_sse(_ptr(Q), _ptr(K), _ptr(LSE), L, N, D, block_len, float(scale), _ptr(s), _ptr(comp),
+                          _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pafu_sse")
 
 
 def pafu_step_indexed(args: CStepArgs) -> None:

@@ -278,6 +278,40 @@ def test_step_indexed_equals_step(w):
     assert torch.equal(A.LSE, B.LSE)
 
 
+# ------------------------------------------------------------- teacher salience (Eq. 4, Eq. 5)
+@pytest.mark.parametrize("L,N,LB", [
+    (700, 2, 200),      # four blocks, the last one half length; every tile ragged
+    (1024, 3, 256),     # blocks that are whole tiles
+    (300, 1, 300),      # a single block
+    (130, 2, 64),       # blocks smaller than a tile
+    (3 * 1560, 2, 1560),  # three frames as blocks: several tiles and key-tile pairs per block
+])
+def test_sse_matches_oracle(L, N, LB):
+    rng = np.random.default_rng(L + N)
+    D = 128
+    # logits with a few dominant keys per row, as attention maps have
+    Q = wl.f32_to_bf16_bits((rng.standard_normal((L, N, D)) * 1.5).astype(np.float32))
+    K = wl.f32_to_bf16_bits((rng.standard_normal((L, N, D)) * 1.5).astype(np.float32))
+    want_s, want_c = oracle.sse(Q, K, LB)
+    dQ, dK = to_device_bf16(Q), to_device_bf16(K)
+    ws = torch.zeros(pafu.pafu_sse_workspace_bytes(L, N, D, LB), dtype=torch.uint8, device="cuda")
+    s = torch.full((L,), float("nan"), device="cuda"); comp = torch.full((3, L), float("nan"), device="cuda")
+    pafu.pafu_sse(dQ, dK, None, LB, 0.0, s, comp, ws)
+    assert pafu.pafu_workspace_status(ws) == 0
+    tol = dict(rtol=1e-3, atol=1e-7)
+    assert np.allclose(comp.cpu().numpy(), want_c, **tol), np.abs(comp.cpu().numpy() - want_c).max()
+    assert np.allclose(s.cpu().numpy(), want_s, **tol)
+    # with the row statistics handed in (as the attention call leaves them) the result is the same
+    shape = pafu.Shape(N, D, None, [0, L])
+    ws2 = torch.zeros(pafu.pafu_workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+    O = torch.empty((L, N, D), dtype=torch.bfloat16, device="cuda"); LSE = torch.empty((N, L), device="cuda")
+    pafu.pafu_chunk_attn(dQ, dK, dK, [0, L], None, None, shape, 0.0, O, LSE, ws2)
+    s2 = torch.full_like(s, float("nan"))
+    pafu.pafu_sse(dQ, dK, LSE, LB, 0.0, s2, None, ws)
+    assert pafu.pafu_workspace_status(ws) == 0
+    assert torch.equal(s, s2)
+
+
 # ---------------------------------------------------------------------------------- step
 @pytest.mark.parametrize("w", SMALL, ids=lambda w: "%s-d%d" % (w.name, w.d_head))
 def test_step_equals_four_calls_and_oracle(w):

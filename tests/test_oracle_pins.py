@@ -325,3 +325,50 @@ def test_sse_against_dense_torch_softmax():
     assert np.allclose(s, want, atol=1e-13)
     # first block has no earlier-block queries, last block no later-block queries
     assert np.all(comp[2, :LB] == 0) and np.all(comp[0, L - LB:] == 0)
+
+
+def test_sse_uniform_attention_closed_form():
+    # zero queries make every row of P uniform (1/L), so each class that has queries gives 1/L:
+    # Eq. 5 then yields 1/L for every key, whichever case applies
+    L, N, D, LB = 30, 3, 4, 7          # last block shorter than the others
+    rng = np.random.default_rng(2)
+    Q = np.zeros((L, N, D), np.uint16)
+    K = bf(rng.standard_normal((L, N, D)).astype(np.float32))
+    s, comp = oracle.sse(Q, K, LB)
+    nb = -(-L // LB)
+    kb = np.arange(L) // LB
+    assert np.allclose(comp[0], np.where(kb < nb - 1, 1.0 / L, 0.0), atol=1e-15)   # later blocks exist
+    assert np.allclose(comp[1], 1.0 / L, atol=1e-15)
+    assert np.allclose(comp[2], np.where(kb > 0, 1.0 / L, 0.0), atol=1e-15)        # earlier blocks exist
+    j = np.arange(L)
+    want = np.where(j < LB, (1 / L + 1 / L) / 2, np.where(j < L - LB, 3 / L / 3, (1 / L + np.where(kb > 0, 1 / L, 0)) / 2))
+    assert np.allclose(s, want, atol=1e-15)
+
+
+def test_sse_brute_force_index_sets():
+    # Eq. 4 written out with explicit index sets I_low(j) = {i | j < l(i)}, I_diag, I_up
+    rng = np.random.default_rng(4)
+    L, N, D, LB = 11, 2, 4, 4
+    Q = bf(rng.standard_normal((L, N, D)).astype(np.float32) * 2)
+    K = bf(rng.standard_normal((L, N, D)).astype(np.float32) * 2)
+    scale = 0.37
+    s, comp = oracle.sse(Q, K, LB, scale=scale)
+    q, k = f32(Q).astype(np.float64), f32(K).astype(np.float64)
+    want = np.zeros((3, L))
+    for n in range(N):
+        P = np.zeros((L, L))
+        for i in range(L):
+            z = np.array([scale * sum(q[i, n, d] * k[j, n, d] for d in range(D)) for j in range(L)])
+            e = np.exp(z - z.max())
+            P[i] = e / e.sum()
+        for j in range(L):
+            lo = lambda i: (i // LB) * LB
+            sets = ([i for i in range(L) if j < lo(i)], [i for i in range(L) if lo(i) <= j < lo(i) + LB],
+                    [i for i in range(L) if j >= lo(i) + LB])
+            for c, I in enumerate(sets):
+                want[c, j] += max((P[i, j] for i in I), default=0.0) / N
+    assert np.allclose(comp, want, atol=1e-14)
+    for j in range(L):
+        w = (want[1, j] + want[0, j]) / 2 if j < LB else ((want[2, j] + want[1, j] + want[0, j]) / 3 if j < L - LB
+                                                            else (want[1, j] + want[2, j]) / 2)
+        assert abs(s[j] - w) < 1e-14
