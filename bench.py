@@ -402,6 +402,41 @@ def run_ours(args):
                "l2": "256 MB written between launches"}
         del flush
 
+    # ---- teacher salience target (Eq. 4, Eq. 5) at the paper's training length: 21 frames of
+    # 1560 tokens, blocks of 4680 (Appendix A).  200 MB of Q and K: larger than L2.
+    sse = None
+    if rank == 0 and w.d_head == 128 and args.sse_tokens > 0:
+        Ls, LBs = args.sse_tokens, wl.CHUNK_TOKENS
+        g = torch.Generator(device="cuda"); g.manual_seed(1)
+        sQ = torch.randn((Ls, w.n_heads, 128), generator=g, device="cuda").to(torch.bfloat16)
+        sK = torch.randn((Ls, w.n_heads, 128), generator=g, device="cuda").to(torch.bfloat16)
+        sws = torch.zeros(pafu.pafu_sse_workspace_bytes(Ls, w.n_heads, 128, LBs), dtype=torch.uint8, device="cuda")
+        s_out = torch.empty(Ls, device="cuda")
+        sLSE = torch.empty((w.n_heads, Ls), device="cuda"); sO = torch.empty_like(sQ)
+        sshape = pafu.Shape(w.n_heads, 128, None, [0, Ls])
+        pafu.pafu_chunk_attn(sQ, sK, sK, [0, Ls], None, None, sshape, 0.0, sO, sLSE, L0.ws)
+        ev_s = [new_events(2) for _ in range(5)]
+        for r in range(7):
+            if r >= 2:
+                ev_s[r - 2][0].record(stream)
+            pafu.pafu_sse(sQ, sK, sLSE, LBs, 0.0, s_out, None, sws)
+            if r >= 2:
+                ev_s[r - 2][1].record(stream)
+        e_f = new_events(2)
+        e_f[0].record(stream)
+        pafu.pafu_sse(sQ, sK, None, LBs, 0.0, s_out, None, sws)
+        e_f[1].record(stream)
+        torch.cuda.synchronize()
+        assert pafu.pafu_workspace_status(sws) == 0
+        s_ms = float(np.median([a.elapsed_time(b) for a, b in ev_s]))
+        s_flops = 2.0 * Ls * Ls * 128 * w.n_heads
+        sse = {"workload": "L = %d tokens, %d heads x 128, blocks of %d" % (Ls, w.n_heads, LBs),
+               "ms_given_lse": s_ms, "TFLOP/s": s_flops / (s_ms * 1e-3) / 1e12,
+               "tensor_frac": s_flops / (s_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+               "peak": "sustained (%.1f)" % peaks["bf16_tflops_sustained"],
+               "ms_with_attention_pass": e_f[0].elapsed_time(e_f[1])}
+        del sQ, sK, sws, sO
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -440,6 +475,7 @@ def run_ours(args):
         },
         "score_qkv": qkv,
         "step_indexed": indexed,
+        "sse": sse,
         "layers_per_step": n_layers,
         "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step / n_layers,
         "peaks": peaks,
@@ -466,6 +502,8 @@ def main():
     ap.add_argument("--layers", type=int, default=1,
                     help="layers per step; 30 with --workload wan1.3b_layer_b25/_b50/_b75 is the full "
                          "denoising step of the 30-layer sweep (every layer has its own cache and head)")
+    ap.add_argument("--sse-tokens", type=int, default=32760,
+                    help="sequence length of the teacher-salience (Eq. 4/5) timing; 0 skips it")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -8,9 +8,9 @@
 //
 // Since exp is monotone, max_i P[i, j] = exp(max_i (z_ij - lse_i)) with lse_i the row's
 // log-sum-exp: given the row statistics (a by-product of the attention kernel) no exponential is
-// needed per element, only one fused multiply-add and one max.  The kernel computes S^T = K Q^T
-// tile by tile (keys are the accumulator's rows, so a thread owns one key and runs its maxima
-// along the columns) and never writes P.
+// needed per element, only one fused multiply-add and one max.  The kernel computes S = Q K^T
+// tile by tile (queries are the accumulator's rows, so -lse is one register per thread, and a
+// thread keeps a running maximum for each of its tile's 128 key columns) and never writes P.
 //
 // Tiling.  Keys and queries are tiled per block of L_B tokens (128 per tile, the last tile of
 // a block ragged), so every (key tile, query tile) pair lies in exactly one class and the class
@@ -20,10 +20,10 @@
 //
 // An item is one head x one pair of key tiles ("slots") x all query tiles; items go to the
 // persistent CTAs round-robin.  Warp roles (320 threads):
-//   warps 0-3  read-out of slot 0 (thread = key row = TMEM lane): t = s * scale*log2e - lse*log2e,
-//              running maximum per class
+//   warps 0-3  read-out of slot 0 (thread = query row = TMEM lane): t = s * scale*log2e - lse*log2e,
+//              running maximum per key column; reduced over the slot's 128 threads per class
 //   warps 4-7  read-out of slot 1
-//   warp  8    MMA issuer: S^T[slot] = K_slot Q_tile^T, M = N = 128, eight K = 16 steps
+//   warp  8    MMA issuer: S[slot] = Q_tile K_slot^T, M = N = 128, eight K = 16 steps
 //   warp  9    TMA loader: the item's K tiles, then Q tiles (+ their 512 bytes of -lse) through a
 //              4-stage ring
 // Tensor memory: 2 slots x 2 accumulator buffers x 128 columns = all 512 columns.
@@ -96,6 +96,16 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return d;
 }
 
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+// barrier among the 128 read-out threads of one slot (hardware barriers 1 and 2)
+__device__ __forceinline__ void slot_barrier(int slot) {
+    asm volatile("bar.sync %0, 128;" ::"r"(slot + 1) : "memory");
+}
+
 // -lse * log2(e) in the padded per-tile layout the main kernel's loader copies.
 __global__ void sse_neglse_kernel(const float* __restrict__ lse, Params p, float* __restrict__ out) {
     grid_dep_wait();
@@ -130,6 +140,7 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
     auto q_empty = [&](int st) { return bar0 + 8 * (12 + kStages + st); };
     __shared__ uint32_t tmem_base_sh;
     __shared__ volatile int abort_flag;
+    __shared__ float red_sh[2 * 4 * kBT];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -207,18 +218,18 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                 for (int g = 0; g < p.n_qt && ok; ++g, ++ring) {
                     const int st = ring % kStages;
                     if (abort_flag || !mbar_wait(q_full(st), (ring / kStages) & 1u)) { fail(512); ok = false; break; }
-                    const uint64_t b = desc0 + ((sQ + st * kStageBytes) >> 4);
+                    const uint64_t b = desc0 + ((sQ + st * kStageBytes) >> 4);       // Q tile
                     for (int s = 0; s < it.n_slots && ok; ++s) {
                         const uint32_t tc = s ? tc1 : tc0;
                         const int buf = tc & 1;
                         if (abort_flag || !mbar_wait(s_empty(s, buf), ((tc >> 1) & 1u) ^ 1u)) { fail(513); ok = false; break; }
                         if (s) ++tc1; else ++tc0;
                         tc_fence_after_sync();
-                        const uint64_t a = desc0 + ((sK + s * kTileBytes) >> 4);
+                        const uint64_t a = desc0 + ((sK + s * kTileBytes) >> 4);     // K tile of this slot
 #pragma unroll
                         for (int kk = 0; kk < kD / 16; ++kk) {
                             const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
-                            umma_ss(tmem + (s * 2 + buf) * kBT, a + off, b + off, idesc, kk > 0);
+                            umma_ss(tmem + (s * 2 + buf) * kBT, b + off, a + off, idesc, kk > 0);   // rows = queries, columns = keys
                         }
                         umma_commit(s_full(s, buf));
                     }
@@ -231,70 +242,96 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
         __syncwarp();
     } else {
         // ------------------------------------------------------------------------ read-out
-        const int slot = warp >> 2;
-        const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
-        const int row_in_tile = (warp & 3) * 32 + lane;
+        // Thread = query row of the streamed tile; it keeps one running maximum per key column
+        // (128 registers) for the class in progress, so the per-row -lse is a register scalar
+        // and each element costs one multiply-add and one max.  When the class changes (the
+        // query tiles pass from earlier blocks to the key's own block to later blocks) and at
+        // the item's end, the 128 threads of the slot reduce their maxima per column and store
+        // them.  The accumulator is read in 16-column pieces, one piece always in flight.
+        const int slot = warp >> 2, wq = warp & 3;
+        const uint32_t lane_base = ((uint32_t)(wq * 32)) << 16;
+        const int t_in_slot = wq * 32 + lane;
+        float* red = red_sh + slot * 4 * kBT;                 // [4 warps][128 columns]
         uint32_t ring = 0, tc = 0;
         bool ok = true;
+        auto wait_warp = [&](uint32_t bar, uint32_t ph, int code) {
+            const bool w = mbar_wait(bar, ph) && !abort_flag;
+            if (!__all_sync(0xffffffffu, w)) { if (lane == 0) fail(code); ok = false; }
+        };
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const Item it = decode_item(p, item);
             const bool active = slot < it.n_slots;
-            float m_low = -INFINITY, m_diag = -INFINITY, m_up = -INFINITY;
+            const int g_diag0 = it.block * p.tpb;                                        // first tile of the key's own block
+            const int g_low0 = it.block == p.n_blocks - 1 ? p.n_qt : g_diag0 + p.tpb;    // first tile of the later blocks
+            float mx[kBT];
+#pragma unroll
+            for (int c = 0; c < kBT; ++c) mx[c] = -INFINITY;
+            // column maxima of the class that just ended -> scratch; classes: 0 low, 1 diag, 2 up
+            auto flush = [&](int cls) {
+                float keep[4];
+#pragma unroll
+                for (int c = 0; c < kBT; ++c) {
+                    const float v = warp_max(mx[c]);
+                    if ((c & 31) == lane) keep[c >> 5] = v;
+                    mx[c] = -INFINITY;
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) red[wq * kBT + k * 32 + lane] = keep[k];
+                slot_barrier(slot);
+                const float v = fmaxf(fmaxf(red[t_in_slot], red[kBT + t_in_slot]),
+                                      fmaxf(red[2 * kBT + t_in_slot], red[3 * kBT + t_in_slot]));
+                const int64_t key = it.key0 + slot * kBT + t_in_slot;
+                if (key < it.block_end) p.M[((int64_t)it.head * 3 + cls) * p.L + key] = v;
+                slot_barrier(slot);
+            };
             for (int g = 0; g < p.n_qt; ++g, ++ring) {
                 const int st = ring % kStages;
-                {
-                    const bool w = mbar_wait(q_full(st), (ring / kStages) & 1u) && !abort_flag;
-                    if (!__all_sync(0xffffffffu, w)) { if (lane == 0) fail(521); ok = false; break; }
-                }
+                wait_warp(q_full(st), (ring / kStages) & 1u, 521);
+                if (!ok) break;
                 if (active) {
+                    if (g == g_diag0 && g > 0) flush(2);
+                    if (g == g_low0) flush(1);
                     const int buf = tc & 1;
-                    {
-                        const bool w = mbar_wait(s_full(slot, buf), (tc >> 1) & 1u) && !abort_flag;
-                        if (!__all_sync(0xffffffffu, w)) { if (lane == 0) fail(522); ok = false; break; }
-                    }
+                    wait_warp(s_full(slot, buf), (tc >> 1) & 1u, 522);
+                    if (!ok) break;
                     ++tc;
                     tc_fence_after_sync();
-                    const float4* nl = reinterpret_cast<const float4*>(smem + 2 * kTileBytes + st * kStageBytes + kTileBytes);
                     const uint32_t tS = tmem + (slot * 2 + buf) * kBT + lane_base;
-                    float tm0 = -INFINITY, tm1 = -INFINITY;
+                    const float nl = reinterpret_cast<const float*>(smem + 2 * kTileBytes + st * kStageBytes + kTileBytes)[t_in_slot];
+                    uint32_t ra[16], rb[16];
+                    PAFU_TMEM_LD_X16(tS, ra);
 #pragma unroll
                     for (int c = 0; c < kBT / 32; ++c) {
-                        uint32_t r[32];
-                        PAFU_TMEM_LD_X32(tS + c * 32, r);
                         tmem_wait_ld();
+                        PAFU_TMEM_LD_X16(tS + c * 32 + 16, rb);
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            const float4 v = nl[c * 8 + q];
-                            const float t0 = fmaf(__uint_as_float(r[4 * q + 0]), p.sl2, v.x);
-                            const float t1 = fmaf(__uint_as_float(r[4 * q + 1]), p.sl2, v.y);
-                            const float t2 = fmaf(__uint_as_float(r[4 * q + 2]), p.sl2, v.z);
-                            const float t3 = fmaf(__uint_as_float(r[4 * q + 3]), p.sl2, v.w);
-                            tm0 = fmax3(tm0, t0, t1);
-                            tm1 = fmax3(tm1, t2, t3);
-                        }
+                        for (int q = 0; q < 16; ++q)
+                            mx[c * 32 + q] = fmaxf(mx[c * 32 + q], fmaf(__uint_as_float(ra[q]), p.sl2, nl));
+                        tmem_wait_ld();
+                        if (c + 1 < kBT / 32) PAFU_TMEM_LD_X16(tS + c * 32 + 32, ra);
+#pragma unroll
+                        for (int q = 0; q < 16; ++q)
+                            mx[c * 32 + 16 + q] = fmaxf(mx[c * 32 + 16 + q], fmaf(__uint_as_float(rb[q]), p.sl2, nl));
                     }
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(s_empty(slot, buf));
-                    const float tm = fmaxf(tm0, tm1);
-                    const int qb = g < (p.n_blocks - 1) * p.tpb ? g / p.tpb : p.n_blocks - 1;
-                    if (qb > it.block) m_low = fmaxf(m_low, tm);
-                    else if (qb == it.block) m_diag = fmaxf(m_diag, tm);
-                    else m_up = fmaxf(m_up, tm);
-                } else {
-                    __syncwarp();
                 }
+                __syncwarp();
                 if (lane == 0) mbar_arrive(q_empty(st));
             }
             if (!ok) break;
             if (active) {
-                const int64_t key = it.key0 + slot * kBT + row_in_tile;
+                // the class in progress at the end, then -inf for the classes that have no queries
+                flush(it.block == p.n_blocks - 1 ? 1 : 0);
+                const int64_t key = it.key0 + slot * kBT + t_in_slot;
                 if (key < it.block_end) {
-                    float* dst = p.M + (int64_t)it.head * 3 * p.L + key;
-                    dst[0] = m_low; dst[p.L] = m_diag; dst[2 * p.L] = m_up;
+                    if (it.block == 0) p.M[((int64_t)it.head * 3 + 2) * p.L + key] = -INFINITY;
+                    if (it.block == p.n_blocks - 1) p.M[((int64_t)it.head * 3 + 0) * p.L + key] = -INFINITY;
                 }
             }
         }
+        if (!ok) tmem_wait_ld();      // no load may be in flight when tensor memory is released
     }
     tc_fence_before_sync();
     __syncthreads();
