@@ -197,6 +197,15 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uin
            ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// Shared-memory matrix descriptor without swizzle, K-major: the operand is stored as core
+// matrices of 8 rows x 16 bytes (128 contiguous bytes each); LBO is the byte distance between
+// core matrices that are neighbours along K, SBO between neighbours along the rows.
+__device__ __forceinline__ uint64_t make_smem_desc_noswizzle(uint32_t smem_addr, uint32_t lbo_bytes,
+                                                             uint32_t sbo_bytes) {
+    return (uint64_t)((smem_addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46);
+}
+
 // ---------------------------------------------------------------- TMEM <-> registers
 // 32x32b shape: the warp touches the 32 lanes of its quadrant (warp_id % 4), thread t owns
 // lane 32 * (warp_id % 4) + t and receives N consecutive 32-bit columns.

@@ -10,7 +10,7 @@ using namespace pafu;
 
 inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 
-// Workspace: [status header][attention scratch][LSE N x L][O L x N x D bf16][-lse padded][maxima].
+// Workspace: [status header][attention scratch][LSE N x L][O L x N x D bf16][queries' extra features][maxima].
 // The attention scratch, LSE and O parts are only used when the caller passes no LSE.
 struct SsePlan {
     size_t attn, lse, o, neglse, maxima, total;
@@ -25,7 +25,7 @@ SsePlan plan(int64_t L, int32_t n_heads, int32_t d_head, int64_t LB) {
     pl.attn = off; off = up256(off + attn_workspace_bytes(st, n_heads, d_head));
     pl.lse = off; off = up256(off + (size_t)n_heads * L * 4);
     pl.o = off; off = up256(off + (size_t)L * n_heads * d_head * 2);
-    pl.neglse = off; off = up256(off + sse_tc::neglse_bytes(p));
+    pl.neglse = off; off = up256(off + sse_tc::aug_bytes(p));
     pl.maxima = off; off = up256(off + sse_tc::maxima_bytes(p));
     pl.total = off;
     return pl;
@@ -70,6 +70,6 @@ extern "C" pafu_status pafu_sse(const uint16_t* Q, const uint16_t* K, const floa
         lse = lse_out;
     }
     return sse_tc::launch(Q, K, lse, L, block_len, n_heads, scale, s, comp,
-                          reinterpret_cast<float*>(base + pl.neglse), reinterpret_cast<float*>(base + pl.maxima),
+                          reinterpret_cast<uint16_t*>(base + pl.neglse), reinterpret_cast<float*>(base + pl.maxima),
                           reinterpret_cast<int*>(base) + kStatusWordTimeout, cs);
 }

@@ -7,25 +7,28 @@
 //   Eq. 5 averages the classes that exist for the key's block.
 //
 // Since exp is monotone, max_i P[i, j] = exp(max_i (z_ij - lse_i)) with lse_i the row's
-// log-sum-exp: given the row statistics (a by-product of the attention kernel) no exponential is
-// needed per element, only one fused multiply-add and one max.  The kernel computes S = Q K^T
-// tile by tile (queries are the accumulator's rows, so -lse is one register per thread, and a
-// thread keeps a running maximum for each of its tile's 128 key columns) and never writes P.
+// log-sum-exp (a by-product of the attention kernel): no exponential is needed per element.
+// The subtraction is folded into the contraction as well: the reduction dimension is extended
+// from 128 to 144, every key gets the extra features (1, 1, 1, 0, ...) and query i the extra
+// features (h, m, l, 0, ...), h + m + l = -lse_i / scale split into three bf16 terms (24 bits),
+// so the accumulator holds q_i.k_j - lse_i / scale and the read-out is a bare running maximum.
+// The kernel computes K Q^T tile by tile (keys are the accumulator's rows: a thread owns one
+// key) and never writes P.
 //
 // Tiling.  Keys and queries are tiled per block of L_B tokens (128 per tile, the last tile of
 // a block ragged), so every (key tile, query tile) pair lies in exactly one class and the class
-// is chosen per tile, not per element.  Columns past a block's end carry -lse = -inf (prepared
-// by a small kernel into a padded [head][query tile][128] array that the loader brings in with
-// the Q tile), rows past the end are not stored.
+// is chosen per tile, not per element.  Query columns past a block's end get -1e30 as their
+// extra feature; key rows past the end are not stored.  The extra features of a query tile are
+// prepared by a small kernel as a 4 KiB block in the operand layout (no swizzle: 8 x 16-byte
+// core matrices) that the loader copies with the tile.
 //
 // An item is one head x one pair of key tiles ("slots") x all query tiles; items go to the
-// persistent CTAs round-robin.  Warp roles (320 threads):
-//   warps 0-3  read-out of slot 0 (thread = query row = TMEM lane): t = s * scale*log2e - lse*log2e,
-//              running maximum per key column; reduced over the slot's 128 threads per class
+// persistent CTAs round-robin.  Warp roles (384 threads):
+//   warps 0-3  read-out of slot 0 (thread = key row = TMEM lane): running maximum per class
 //   warps 4-7  read-out of slot 1
-//   warp  8    MMA issuer: S[slot] = Q_tile K_slot^T, M = N = 128, eight K = 16 steps
-//   warp  9    TMA loader: the item's K tiles, then Q tiles (+ their 512 bytes of -lse) through a
-//              4-stage ring
+//   warps 8,10 MMA issuers, one per slot: S[slot] = K_slot Q_tile^T, M = N = 128, nine K = 16 steps
+//   warp  9    TMA loader: the item's K tiles, then Q tiles (+ extra features) through a 4-stage ring
+//   warp  11   idle
 // Tensor memory: 2 slots x 2 accumulator buffers x 128 columns = all 512 columns.
 // The per-head maxima go to scratch [head][class][key] in the log2 domain; a last kernel takes
 // exp2, averages over heads in head order and applies Eq. 5.  Every mbarrier wait is bounded.
@@ -41,12 +44,13 @@ using namespace sm100;
 constexpr int kD = 128;
 constexpr int kBT = 128;                       // tokens per tile, keys and queries alike
 constexpr int kStages = 4;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;
 constexpr int kTileBytes = kBT * kD * 2;       // 32 KiB
 constexpr int kHalfBytes = kTileBytes / 2;     // one [128 rows x 64 cols] swizzled half
-constexpr int kLseBytes = kBT * 4;
-constexpr int kStageBytes = kTileBytes + 1024; // Q tile, then -lse (padded to keep 1 KiB alignment)
-constexpr int kSmemBytes = 2 * kTileBytes + kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int kAugBytes = kBT * 16 * 2;        // 4 KiB: 16 extra reduction columns of one tile
+constexpr int kStageBytes = kTileBytes + kAugBytes;   // Q tile, then its extra features
+constexpr int kSmemBytes = 2 * kTileBytes + kAugBytes + kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr float kMasked = -1.0e30f;            // extra feature of a query column that does not exist
 
 struct Params {
     int64_t L, LB;
@@ -56,7 +60,8 @@ struct Params {
     int pairs, pairs_last;    // key-tile pairs per block
     int items_per_head;       // (n_blocks - 1) * pairs + pairs_last
     float sl2;                // scale * log2(e)
-    const float* neg_lse2;    // [n_heads][n_qt][128]: -lse * log2(e), -inf on padding
+    float inv_scale;
+    const uint16_t* q_aug;    // [n_heads][n_qt][2048] bf16: extra features per query tile, operand layout
     float* M;                 // [n_heads][3][L]: per-head class maxima, log2 domain
     int* status;
 };
@@ -96,30 +101,43 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return d;
 }
 
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
+__device__ __forceinline__ uint16_t bf16_rne(float x) {
+    const uint32_t u = __float_as_uint(x);
+    return (uint16_t)((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
 }
-// barrier among the 128 read-out threads of one slot (hardware barriers 1 and 2)
-__device__ __forceinline__ void slot_barrier(int slot) {
-    asm volatile("bar.sync %0, 128;" ::"r"(slot + 1) : "memory");
-}
+__device__ __forceinline__ float bf16_val(uint16_t b) { return __uint_as_float(((uint32_t)b) << 16); }
 
-// -lse * log2(e) in the padded per-tile layout the main kernel's loader copies.
-__global__ void sse_neglse_kernel(const float* __restrict__ lse, Params p, float* __restrict__ out) {
+// Extra features of every query tile in the operand's shared-memory layout (K-major, no
+// swizzle): element (row r, column c) of a [128 x 16] tile sits at byte
+// (r / 8) * 256 + (c / 8) * 128 + (r % 8) * 16 + (c % 8) * 2.  Columns 0..2 carry the three
+// bf16 terms of -lse / scale, the rest are zero.
+__global__ void sse_aug_kernel(const float* __restrict__ lse, Params p, uint16_t* __restrict__ out) {
     grid_dep_wait();
-    const int64_t n = (int64_t)p.n_heads * p.n_qt * kBT;
+    const int64_t n = (int64_t)p.n_heads * p.n_qt * (kAugBytes / 2);
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % kBT);
-        const int g = (int)((i / kBT) % p.n_qt);
-        const int head = (int)(i / ((int64_t)kBT * p.n_qt));
-        int qb; int64_t row;
-        decode_qtile(p, g, qb, row);
-        const int64_t e = (int64_t)(qb + 1) * p.LB;
-        const int64_t end = e < p.L ? e : p.L;
-        const int64_t q = row + c;
-        out[i] = q < end ? -lse[(int64_t)head * p.L + q] * 1.4426950408889634f : -INFINITY;
+        const int e = (int)(i % (kAugBytes / 2));
+        const int g = (int)((i / (kAugBytes / 2)) % p.n_qt);
+        const int head = (int)(i / ((int64_t)(kAugBytes / 2) * p.n_qt));
+        const int r = (e / 128) * 8 + (e % 64) / 8;
+        const int c = ((e % 128) / 64) * 8 + e % 8;
+        uint16_t v = 0;
+        if (c < 3) {
+            int qb; int64_t row;
+            decode_qtile(p, g, qb, row);
+            const int64_t end_b = (int64_t)(qb + 1) * p.LB;
+            const int64_t end = end_b < p.L ? end_b : p.L;
+            const int64_t q = row + r;
+            if (q < end) {
+                const float a = -lse[(int64_t)head * p.L + q] * p.inv_scale;
+                const uint16_t h = bf16_rne(a);
+                const uint16_t m = bf16_rne(a - bf16_val(h));
+                const uint16_t l = bf16_rne(a - bf16_val(h) - bf16_val(m));
+                v = c == 0 ? h : (c == 1 ? m : l);
+            } else {
+                v = c == 0 ? bf16_rne(kMasked) : (uint16_t)0;
+            }
+        }
+        out[i] = v;
     }
 }
 
@@ -129,8 +147,9 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sK = smem_u32(smem);                     // 2 slots x 32 KiB
-    const uint32_t sQ = sK + 2 * kTileBytes;                // ring of {Q tile, -lse}
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kTileBytes + kStages * kStageBytes);
+    const uint32_t sKaug = sK + 2 * kTileBytes;             // the keys' extra features (1, 1, 1, 0, ...)
+    const uint32_t sQ = sKaug + kAugBytes;                  // ring of {Q tile, its extra features}
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * kTileBytes + kAugBytes + kStages * kStageBytes);
     const uint32_t bar0 = smem_u32(bars);
     auto k_full = [&](int s) { return bar0 + 8 * (0 + s); };
     auto k_empty = [&](int s) { return bar0 + 8 * (2 + s); };
@@ -140,7 +159,6 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
     auto q_empty = [&](int st) { return bar0 + 8 * (12 + kStages + st); };
     __shared__ uint32_t tmem_base_sh;
     __shared__ volatile int abort_flag;
-    __shared__ float red_sh[2 * 4 * kBT];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -150,12 +168,23 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
         }
         for (int st = 0; st < kStages; ++st) {
             mbar_init(q_full(st), 1);
-            mbar_init(q_empty(st), 1 + 8);      // the issuer's commit and every read-out warp
+            mbar_init(q_empty(st), 2);          // both issuers release a stage
         }
         abort_flag = 0;
         fence_barrier_init();
     }
     if (warp == 8) { tmem_alloc(smem_u32(&tmem_base_sh), 512); tmem_relinquish(); }
+    // the keys' extra features are the same for every tile: ones in columns 0..2 of each row
+    for (int w = tid; w < kAugBytes / 4; w += kThreads) {
+        const int off = w * 4, in_group = off % 256;
+        uint32_t v = 0;
+        if (in_group < 128) {                       // columns 0..7
+            const int pair = (in_group % 16) / 4;   // columns 2 * pair, 2 * pair + 1
+            v = pair == 0 ? 0x3f803f80u : (pair == 1 ? 0x00003f80u : 0u);
+        }
+        reinterpret_cast<uint32_t*>(smem + 2 * kTileBytes)[w] = v;
+    }
+    fence_proxy_async_smem();                       // the tensor core reads it through the async proxy
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -190,10 +219,10 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                     int qb; int64_t row;
                     decode_qtile(p, g, qb, row);
                     const uint32_t dst = sQ + st * kStageBytes;
-                    mbar_arrive_expect_tx(q_full(st), kTileBytes + kLseBytes);
+                    mbar_arrive_expect_tx(q_full(st), kTileBytes + kAugBytes);
                     tma_load_3d(dst, &mQ, q_full(st), 0, it.head, (int)row);
                     tma_load_3d(dst + kHalfBytes, &mQ, q_full(st), 64, it.head, (int)row);
-                    bulk_load(dst + kTileBytes, p.neg_lse2 + ((int64_t)it.head * p.n_qt + g) * kBT, kLseBytes, q_full(st));
+                    bulk_load(dst + kTileBytes, p.q_aug + ((int64_t)it.head * p.n_qt + g) * (kAugBytes / 2), kAugBytes, q_full(st));
                 }
             }
             if (!ok)
@@ -201,134 +230,124 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                     mbar_wait(q_full(r % kStages), (r / kStages) & 1u);
         }
         __syncwarp();
-    } else if (warp == 8) {
-        // ---------------------------------------------------------------------- MMA issuer
+    } else if (warp == 11) {
+        // idle: completes the third warpgroup
+    } else if (warp >= 8) {
+        // ------------------------------------------- MMA issuers: warp 8 -> slot 0, warp 10 -> slot 1
+        // One issuing thread per slot: with the waits, commits and descriptor arithmetic of its
+        // loop a single thread issues roughly one tcgen05.mma per 100 clocks, less than the tensor
+        // core consumes (a 128 x 128 x 16 step takes 64).
         if (elect_one()) {
+            const int slot = warp == 8 ? 0 : 1;
             const uint32_t idesc = make_idesc_bf16(kBT, kBT, false, false);
             const uint64_t desc0 = make_smem_desc_sw128(0, 16, 1024);
-            uint32_t ring = 0, kc0 = 0, kc1 = 0, tc0 = 0, tc1 = 0;
+            // extra features: no swizzle, core matrices 128 bytes apart along K, 256 along rows
+            const uint64_t desc_aug = make_smem_desc_noswizzle(0, 128, 256);
+            const uint64_t a_aug = desc_aug + (sKaug >> 4);
+            const uint64_t a = desc0 + ((sK + slot * kTileBytes) >> 4);     // K tile of this slot
+            uint32_t ring = 0, kc = 0, tc = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                 const Item it = decode_item(p, item);
-                for (int s = 0; s < it.n_slots && ok; ++s) {
-                    const uint32_t kc = s ? kc1 : kc0;
-                    if (abort_flag || !mbar_wait(k_full(s), kc & 1u)) { fail(511); ok = false; break; }
-                    if (s) ++kc1; else ++kc0;
+                const bool active = slot < it.n_slots;
+                if (active) {
+                    if (abort_flag || !mbar_wait(k_full(slot), kc & 1u)) { fail(511); ok = false; break; }
+                    ++kc;
                 }
                 for (int g = 0; g < p.n_qt && ok; ++g, ++ring) {
                     const int st = ring % kStages;
                     if (abort_flag || !mbar_wait(q_full(st), (ring / kStages) & 1u)) { fail(512); ok = false; break; }
+                    if (!active) { mbar_arrive(q_empty(st)); continue; }    // a stage is released by both issuers
+                    const int buf = tc & 1;
+                    if (abort_flag || !mbar_wait(s_empty(slot, buf), ((tc >> 1) & 1u) ^ 1u)) { fail(513); ok = false; break; }
+                    ++tc;
+                    tc_fence_after_sync();
                     const uint64_t b = desc0 + ((sQ + st * kStageBytes) >> 4);       // Q tile
-                    for (int s = 0; s < it.n_slots && ok; ++s) {
-                        const uint32_t tc = s ? tc1 : tc0;
-                        const int buf = tc & 1;
-                        if (abort_flag || !mbar_wait(s_empty(s, buf), ((tc >> 1) & 1u) ^ 1u)) { fail(513); ok = false; break; }
-                        if (s) ++tc1; else ++tc0;
-                        tc_fence_after_sync();
-                        const uint64_t a = desc0 + ((sK + s * kTileBytes) >> 4);     // K tile of this slot
+                    const uint64_t b_aug = desc_aug + ((sQ + st * kStageBytes + kTileBytes) >> 4);
+                    const uint32_t d = tmem + (slot * 2 + buf) * kBT;
 #pragma unroll
-                        for (int kk = 0; kk < kD / 16; ++kk) {
-                            const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
-                            umma_ss(tmem + (s * 2 + buf) * kBT, b + off, a + off, idesc, kk > 0);   // rows = queries, columns = keys
-                        }
-                        umma_commit(s_full(s, buf));
+                    for (int kk = 0; kk < kD / 16; ++kk) {
+                        const uint32_t off = ((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4;
+                        umma_ss(d, a + off, b + off, idesc, kk > 0);                 // rows = keys, columns = queries
                     }
-                    if (ok) umma_commit(q_empty(st));
+                    umma_ss(d, a_aug, b_aug, idesc, 1);                              // ... - lse / scale
+                    umma_commit(s_full(slot, buf));
+                    umma_commit(q_empty(st));
                 }
-                if (ok)
-                    for (int s = 0; s < it.n_slots; ++s) umma_commit(k_empty(s));
+                if (ok && active) umma_commit(k_empty(slot));
             }
         }
         __syncwarp();
     } else {
         // ------------------------------------------------------------------------ read-out
-        // Thread = query row of the streamed tile; it keeps one running maximum per key column
-        // (128 registers) for the class in progress, so the per-row -lse is a register scalar
-        // and each element costs one multiply-add and one max.  When the class changes (the
-        // query tiles pass from earlier blocks to the key's own block to later blocks) and at
-        // the item's end, the 128 threads of the slot reduce their maxima per column and store
-        // them.  The accumulator is read in 16-column pieces, one piece always in flight.
-        const int slot = warp >> 2, wq = warp & 3;
-        const uint32_t lane_base = ((uint32_t)(wq * 32)) << 16;
-        const int t_in_slot = wq * 32 + lane;
-        float* red = red_sh + slot * 4 * kBT;                 // [4 warps][128 columns]
-        uint32_t ring = 0, tc = 0;
+        // Thread = key row.  The accumulator already holds q.k - lse / scale, so a tile costs
+        // each thread 128 values and 64 three-way maxima.  It is read in two halves of 64
+        // columns into two register sets: half 1 loads during the arithmetic on half 0, half 0
+        // of the next tile during the arithmetic on half 1, and the buffer goes back to the
+        // issuer as soon as its second half has landed.
+        const int slot = warp >> 2;
+        const uint32_t lane_base = ((uint32_t)((warp & 3) * 32)) << 16;
+        const int row_in_tile = (warp & 3) * 32 + lane;
+        uint32_t tc = 0;
         bool ok = true;
         auto wait_warp = [&](uint32_t bar, uint32_t ph, int code) {
             const bool w = mbar_wait(bar, ph) && !abort_flag;
             if (!__all_sync(0xffffffffu, w)) { if (lane == 0) fail(code); ok = false; }
         };
+        auto max64 = [&](const uint32_t (&r)[64], float& tm0, float& tm1) {
+#pragma unroll
+            for (int q = 0; q < 16; ++q) {
+                tm0 = fmax3(tm0, __uint_as_float(r[4 * q + 0]), __uint_as_float(r[4 * q + 1]));
+                tm1 = fmax3(tm1, __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+            }
+        };
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const Item it = decode_item(p, item);
-            const bool active = slot < it.n_slots;
-            const int g_diag0 = it.block * p.tpb;                                        // first tile of the key's own block
-            const int g_low0 = it.block == p.n_blocks - 1 ? p.n_qt : g_diag0 + p.tpb;    // first tile of the later blocks
-            float mx[kBT];
-#pragma unroll
-            for (int c = 0; c < kBT; ++c) mx[c] = -INFINITY;
-            // column maxima of the class that just ended -> scratch; classes: 0 low, 1 diag, 2 up
-            auto flush = [&](int cls) {
-                float keep[4];
-#pragma unroll
-                for (int c = 0; c < kBT; ++c) {
-                    const float v = warp_max(mx[c]);
-                    if ((c & 31) == lane) keep[c >> 5] = v;
-                    mx[c] = -INFINITY;
-                }
-#pragma unroll
-                for (int k = 0; k < 4; ++k) red[wq * kBT + k * 32 + lane] = keep[k];
-                slot_barrier(slot);
-                const float v = fmaxf(fmaxf(red[t_in_slot], red[kBT + t_in_slot]),
-                                      fmaxf(red[2 * kBT + t_in_slot], red[3 * kBT + t_in_slot]));
-                const int64_t key = it.key0 + slot * kBT + t_in_slot;
-                if (key < it.block_end) p.M[((int64_t)it.head * 3 + cls) * p.L + key] = v;
-                slot_barrier(slot);
-            };
-            for (int g = 0; g < p.n_qt; ++g, ++ring) {
-                const int st = ring % kStages;
-                wait_warp(q_full(st), (ring / kStages) & 1u, 521);
-                if (!ok) break;
-                if (active) {
-                    if (g == g_diag0 && g > 0) flush(2);
-                    if (g == g_low0) flush(1);
-                    const int buf = tc & 1;
-                    wait_warp(s_full(slot, buf), (tc >> 1) & 1u, 522);
-                    if (!ok) break;
-                    ++tc;
-                    tc_fence_after_sync();
-                    const uint32_t tS = tmem + (slot * 2 + buf) * kBT + lane_base;
-                    const float nl = reinterpret_cast<const float*>(smem + 2 * kTileBytes + st * kStageBytes + kTileBytes)[t_in_slot];
-                    uint32_t ra[16], rb[16];
-                    PAFU_TMEM_LD_X16(tS, ra);
-#pragma unroll
-                    for (int c = 0; c < kBT / 32; ++c) {
-                        tmem_wait_ld();
-                        PAFU_TMEM_LD_X16(tS + c * 32 + 16, rb);
-#pragma unroll
-                        for (int q = 0; q < 16; ++q)
-                            mx[c * 32 + q] = fmaxf(mx[c * 32 + q], fmaf(__uint_as_float(ra[q]), p.sl2, nl));
-                        tmem_wait_ld();
-                        if (c + 1 < kBT / 32) PAFU_TMEM_LD_X16(tS + c * 32 + 32, ra);
-#pragma unroll
-                        for (int q = 0; q < 16; ++q)
-                            mx[c * 32 + 16 + q] = fmaxf(mx[c * 32 + 16 + q], fmaf(__uint_as_float(rb[q]), p.sl2, nl));
-                    }
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(s_empty(slot, buf));
-                }
+            if (slot >= it.n_slots) continue;
+            float m_low = -INFINITY, m_diag = -INFINITY, m_up = -INFINITY;
+            uint32_t ra[64], rb[64];
+            wait_warp(s_full(slot, tc & 1), (tc >> 1) & 1u, 522);
+            if (!ok) break;
+            tc_fence_after_sync();
+            {
+                const uint32_t tS = tmem + (slot * 2 + (tc & 1)) * kBT + lane_base;
+                PAFU_TMEM_LD_X32(tS, ra);
+                PAFU_TMEM_LD_X32(tS + 32, ra + 32);
+            }
+            for (int g = 0; g < p.n_qt; ++g) {
+                const int buf = tc & 1;
+                const uint32_t tS = tmem + (slot * 2 + buf) * kBT + lane_base;
+                float tm0 = -INFINITY, tm1 = -INFINITY;
+                tmem_wait_ld();                                   // half 0 in ra
+                PAFU_TMEM_LD_X32(tS + 64, rb);
+                PAFU_TMEM_LD_X32(tS + 96, rb + 32);
+                max64(ra, tm0, tm1);
+                tmem_wait_ld();                                   // half 1 in rb: the buffer is free
+                tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(q_empty(st));
+                if (lane == 0) mbar_arrive(s_empty(slot, buf));
+                ++tc;
+                if (g + 1 < p.n_qt) {
+                    wait_warp(s_full(slot, tc & 1), (tc >> 1) & 1u, 523);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t tN = tmem + (slot * 2 + (tc & 1)) * kBT + lane_base;
+                    PAFU_TMEM_LD_X32(tN, ra);
+                    PAFU_TMEM_LD_X32(tN + 32, ra + 32);
+                }
+                max64(rb, tm0, tm1);
+                const float tm = fmaxf(tm0, tm1);
+                const int qb = g < (p.n_blocks - 1) * p.tpb ? g / p.tpb : p.n_blocks - 1;
+                if (qb > it.block) m_low = fmaxf(m_low, tm);
+                else if (qb == it.block) m_diag = fmaxf(m_diag, tm);
+                else m_up = fmaxf(m_up, tm);
             }
             if (!ok) break;
-            if (active) {
-                // the class in progress at the end, then -inf for the classes that have no queries
-                flush(it.block == p.n_blocks - 1 ? 1 : 0);
-                const int64_t key = it.key0 + slot * kBT + t_in_slot;
-                if (key < it.block_end) {
-                    if (it.block == 0) p.M[((int64_t)it.head * 3 + 2) * p.L + key] = -INFINITY;
-                    if (it.block == p.n_blocks - 1) p.M[((int64_t)it.head * 3 + 0) * p.L + key] = -INFINITY;
-                }
+            const int64_t key = it.key0 + slot * kBT + row_in_tile;
+            if (key < it.block_end) {
+                // log2 domain; a class without queries stays -inf, a masked column gives about -1e29
+                float* dst = p.M + (int64_t)it.head * 3 * p.L + key;
+                dst[0] = m_low * p.sl2; dst[p.L] = m_diag * p.sl2; dst[2 * p.L] = m_up * p.sl2;
             }
         }
         if (!ok) tmem_wait_ld();      // no load may be in flight when tensor memory is released
@@ -370,18 +389,19 @@ inline Params make_params(int64_t L, int64_t LB, int n_heads, float scale) {
     p.pairs_last = (p.tpb_last + 1) / 2;
     p.items_per_head = (p.n_blocks - 1) * p.pairs + p.pairs_last;
     p.sl2 = scale * 1.4426950408889634f;
-    p.neg_lse2 = nullptr; p.M = nullptr; p.status = nullptr;
+    p.inv_scale = 1.0f / scale;
+    p.q_aug = nullptr; p.M = nullptr; p.status = nullptr;
     return p;
 }
 
-inline size_t neglse_bytes(const Params& p) { return (size_t)p.n_heads * p.n_qt * kBT * 4; }
+inline size_t aug_bytes(const Params& p) { return (size_t)p.n_heads * p.n_qt * kAugBytes; }
 inline size_t maxima_bytes(const Params& p) { return (size_t)p.n_heads * 3 * p.L * 4; }
 
 inline pafu_status launch(const uint16_t* Q, const uint16_t* K, const float* lse, int64_t L, int64_t LB,
-                          int n_heads, float scale, float* s, float* comp, float* neg_lse2, float* M,
+                          int n_heads, float scale, float* s, float* comp, uint16_t* q_aug, float* M,
                           int* status, cudaStream_t stream) {
     Params p = make_params(L, LB, n_heads, scale);
-    p.neg_lse2 = neg_lse2; p.M = M; p.status = status;
+    p.q_aug = q_aug; p.M = M; p.status = status;
     CUtensorMap mQ, mK;
     if (!TmapEncoder::token_tensor(&mQ, Q, (uint64_t)L, n_heads, kD, kBT) ||
         !TmapEncoder::token_tensor(&mK, K, (uint64_t)L, n_heads, kD, kBT)) return PAFU_ERR_CUDA;
@@ -392,9 +412,9 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* K, const float* lse
         attr_set = true;
     }
     const int sms = device_sm_count();
-    const int64_t n_pad = (int64_t)n_heads * p.n_qt * kBT;
-    const int g0 = (int)((n_pad + 255) / 256 < 4 * sms ? (n_pad + 255) / 256 : 4 * sms);
-    if (launch_dependent(sse_neglse_kernel, dim3(g0), dim3(256), 0, stream, 1, lse, p, neg_lse2) != cudaSuccess)
+    const int64_t n_pad = (int64_t)n_heads * p.n_qt * (kAugBytes / 2);
+    const int g0 = (int)((n_pad + 255) / 256 < 8 * sms ? (n_pad + 255) / 256 : 8 * sms);
+    if (launch_dependent(sse_aug_kernel, dim3(g0), dim3(256), 0, stream, 1, lse, p, q_aug) != cudaSuccess)
         return PAFU_ERR_CUDA;
     const int n_items = n_heads * p.items_per_head;
     const int grid = n_items < sms ? n_items : sms;
