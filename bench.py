@@ -402,6 +402,28 @@ def run_ours(args):
                "l2": "256 MB written between launches"}
         del flush
 
+    # ---- the paper's own schedule for pruning (Sec. 3.3): one Top-k at the final layer, its indices
+    # applied to all 30 layers' caches in one launch (30 x 172.5 MB moved: far larger than L2)
+    shared = None
+    if rank == 0 and args.shared_layers > 0:
+        nl = args.shared_layers
+        Ks = [torch.empty_like(L0.K).copy_(L0.K) for _ in range(nl)]; Vs = [torch.empty_like(L0.V).copy_(L0.V) for _ in range(nl)]
+        Kcs = [torch.empty_like(L0.Kc) for _ in range(nl)]; Vcs = [torch.empty_like(L0.Vc) for _ in range(nl)]
+        ev_c = [new_events(2) for _ in range(5)]
+        for r in range(7):
+            if r >= 2:
+                ev_c[r - 2][0].record(stream)
+            pafu.pafu_select(L0.scores, L0.shape, L0.policy, L0.idx, L0.ws)
+            pafu.pafu_compact_layers(Ks, Vs, L0.scores, L0.idx, L0.shape, L0.policy, Kcs, Vcs, L0.SLc)
+            if r >= 2:
+                ev_c[r - 2][1].record(stream)
+        torch.cuda.synchronize()
+        c_ms = float(np.median([a.elapsed_time(b) for a, b in ev_c]))
+        c_bytes = nl * (work["compact_bytes"] - L0.nB * 4) + work["select_bytes"] + L0.nB * 8
+        shared = {"workload": "one select + one %d-layer compaction with shared indices" % nl, "ms": c_ms,
+                  "GB/s": c_bytes / (c_ms * 1e-3) / 1e9, "hbm_frac": c_bytes / (c_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        del Ks, Vs, Kcs, Vcs
+
     # ---- teacher salience target (Eq. 4, Eq. 5) at the paper's training length: 21 frames of
     # 1560 tokens, blocks of 4680 (Appendix A).  200 MB of Q and K: larger than L2.
     sse = None
@@ -477,6 +499,7 @@ def run_ours(args):
         "score_qkv": qkv,
         "step_indexed": indexed,
         "sse": sse,
+        "shared_index_compaction": shared,
         "layers_per_step": n_layers,
         "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step / n_layers,
         "peaks": peaks,
@@ -503,6 +526,8 @@ def main():
     ap.add_argument("--layers", type=int, default=1,
                     help="layers per step; 30 with --workload wan1.3b_layer_b25/_b50/_b75 is the full "
                          "denoising step of the 30-layer sweep (every layer has its own cache and head)")
+    ap.add_argument("--shared-layers", type=int, default=30,
+                    help="layers pruned with one shared index list in the shared-index timing; 0 skips it")
     ap.add_argument("--sse-tokens", type=int, default=32760,
                     help="sequence length of the teacher-salience (Eq. 4/5) timing; 0 skips it")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

@@ -40,6 +40,7 @@ extern "C" {
 #endif
 
 #define PAFU_MAX_STREAMS 32
+#define PAFU_MAX_LAYERS 64
 
 typedef int32_t pafu_status;
 enum {
@@ -167,6 +168,18 @@ pafu_status pafu_select(const float* scores, const pafu_shape* shape, const pafu
 pafu_status pafu_compact(const uint16_t* K, const uint16_t* V, const float* SL, const int32_t* idx,
                          const pafu_shape* shape, const pafu_policy* policy,
                          uint16_t* Kc, uint16_t* Vc, float* SLc, void* stream);
+
+/* Step 3 for every layer at once.  The paper scores and selects at the final layer only and
+ * reuses the indices for all layers (Sec. 3.3: the Top-k sets of the layers agree at t_0; Sec. 3.4:
+ * the head sits in the final layer), so one index list prunes n_layers caches.  Exactly
+ * pafu_compact applied to each (K[l], V[l]) -> (Kc[l], Vc[l]) with the same idx, in one launch;
+ * SL -> SLc (both or neither NULL) is compacted once.
+ *   K, V, Kc, Vc   HOST arrays of n_layers DEVICE pointers (read before the call returns), each
+ *                  tensor laid out as for pafu_compact; n_layers <= PAFU_MAX_LAYERS */
+pafu_status pafu_compact_layers(const uint16_t* const* K, const uint16_t* const* V, int32_t n_layers,
+                                const float* SL, const int32_t* idx, const pafu_shape* shape,
+                                const pafu_policy* policy, uint16_t* const* Kc, uint16_t* const* Vc,
+                                float* SLc, void* stream);
 
 /* Step 4 - chunk attention over the retained cache (Sec. 3.2 for the operator
  * P = softmax(Q K^T / sqrt(D)); Eq. 2 / Eq. 7 for what it ranges over).

@@ -29,7 +29,7 @@ STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET
 EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
            "pafu_workspace_status", "pafu_score", "pafu_score_qkv", "pafu_select", "pafu_compact",
            "pafu_chunk_attn", "pafu_chunk_attn_indexed", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_indexed", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host",
-           "pafu_sse_workspace_bytes", "pafu_sse"]
+           "pafu_sse_workspace_bytes", "pafu_sse", "pafu_compact_layers"]
 
 
 class PafuError(RuntimeError):
@@ -112,6 +112,9 @@ def lib() -> ctypes.CDLL:
                                               ctypes.c_float, vp, vp, vp, sz, vp]
         L.pafu_step_indexed.restype = i32
         L.pafu_step_indexed.argtypes = [ctypes.POINTER(CStepArgs), vp]
+        L.pafu_compact_layers.restype = i32
+        L.pafu_compact_layers.argtypes = [vp, vp, i32, vp, vp, ctypes.POINTER(CShape), ctypes.POINTER(CPolicy),
+                                          vp, vp, vp, vp]
         L.pafu_sse_workspace_bytes.restype = sz
         L.pafu_sse_workspace_bytes.argtypes = [i64, i32, i32, i64]
         L.pafu_sse.restype = i32
@@ -240,6 +243,14 @@ def pafu_select(scores: torch.Tensor, shape: Shape, policy, idx: torch.Tensor,
 def pafu_compact(K, V, SL, idx, shape: Shape, policy, Kc, Vc, SLc) -> None:
     _check(lib().pafu_compact(_ptr(K), _ptr(V), _ptr(SL), _ptr(idx), ctypes.byref(shape.c), policy,
                               _ptr(Kc), _ptr(Vc), _ptr(SLc), _stream()), "pafu_compact")
+
+
+def pafu_compact_layers(Ks, Vs, SL, idx, shape: Shape, policy, Kcs, Vcs, SLc) -> None:
+    """One index list applied to every layer's cache (lists of per-layer tensors)."""
+    n = len(Ks)
+    arr = lambda ts: (ctypes.c_void_p * max(n, 1))(*[_ptr(t) for t in ts])
+    _check(lib().pafu_compact_layers(arr(Ks), arr(Vs), n, _ptr(SL), _ptr(idx), ctypes.byref(shape.c), policy,
+                                     arr(Kcs), arr(Vcs), _ptr(SLc), _stream()), "pafu_compact_layers")
 
 
 def pafu_chunk_attn(Q, Kc, Vc, cu_B, Kq, Vq, shape: Shape, scale: float, O, LSE=None,

@@ -206,6 +206,34 @@ pafu_status pafu_compact(const uint16_t* K, const uint16_t* V, const float* SL, 
     return launch_compact(K, V, SL, idx, st, (int32_t)dm, Kc, Vc, SLc, static_cast<cudaStream_t>(stream));
 }
 
+pafu_status pafu_compact_layers(const uint16_t* const* K, const uint16_t* const* V, int32_t n_layers,
+                                const float* SL, const int32_t* idx, const pafu_shape* shape,
+                                const pafu_policy* policy, uint16_t* const* Kc, uint16_t* const* Vc,
+                                float* SLc, void* stream) {
+    pafu_status e = shape_ok(shape, true, false);
+    if (e != PAFU_OK) return e;
+    if (n_layers < 0) return PAFU_ERR_INVALID_ARG;
+    if (n_layers > PAFU_MAX_LAYERS) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    const int64_t dm = (int64_t)shape->n_heads * shape->d_head;
+    if (dm % 8 != 0 || dm > 0x7fffffffLL) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    StreamTable st;
+    memset(&st, 0, sizeof st);
+    st.n_streams = shape->n_streams;
+    fill_prefix(st.cu_T, shape->cu_T, shape->n_streams);
+    e = fill_policy(shape, policy, &st);
+    if (e != PAFU_OK) return e;
+    if (st.cu_B[st.n_streams] == 0 || n_layers == 0) return PAFU_OK;
+    if (K == nullptr || V == nullptr || Kc == nullptr || Vc == nullptr || idx == nullptr) return PAFU_ERR_INVALID_ARG;
+    if ((SL == nullptr) != (SLc == nullptr)) return PAFU_ERR_INVALID_ARG;
+    if (!aligned16(idx)) return PAFU_ERR_MISALIGNED;
+    for (int l = 0; l < n_layers; ++l) {
+        if (K[l] == nullptr || V[l] == nullptr || Kc[l] == nullptr || Vc[l] == nullptr) return PAFU_ERR_INVALID_ARG;
+        if (!aligned16(K[l]) || !aligned16(V[l]) || !aligned16(Kc[l]) || !aligned16(Vc[l])) return PAFU_ERR_MISALIGNED;
+        if (Kc[l] == K[l] || Vc[l] == V[l] || Kc[l] == V[l] || Vc[l] == K[l]) return PAFU_ERR_INVALID_ARG;
+    }
+    return launch_compact_layers(K, V, n_layers, SL, idx, st, (int32_t)dm, Kc, Vc, SLc, static_cast<cudaStream_t>(stream));
+}
+
 pafu_status pafu_chunk_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
                             const int64_t* cu_B, const uint16_t* Kq, const uint16_t* Vq,
                             const pafu_shape* shape, float scale, uint16_t* O, float* LSE,

@@ -83,6 +83,9 @@ pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* i
 pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL,
                            const int32_t* idx, const StreamTable& st, int32_t d_model,
                            uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream);
+pafu_status launch_compact_layers(const uint16_t* const* K, const uint16_t* const* V, int32_t n_layers,
+                                  const float* SL, const int32_t* idx, const StreamTable& st, int32_t d_model,
+                                  uint16_t* const* Kc, uint16_t* const* Vc, float* SLc, cudaStream_t stream);
 pafu_status launch_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
                         const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
                         int32_t n_heads, int32_t d_head, float scale, uint16_t* O, float* LSE,

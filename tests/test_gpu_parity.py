@@ -219,6 +219,73 @@ def test_attention_segment_edge_cases():
             close(LSE.cpu().numpy(), wl_, "edge LSE")
 
 
+# ------------------------------------------------- one index list for all layers; Algorithm 2
+def test_algorithm2_cache_update_over_chunks():
+    """Algorithm 2 run chunk by chunk: the S-MLP scores the new chunk's [q, k, v] at the final
+    layer, the salience list SL is carried with the cache, and when the cache would overflow the
+    Top-k of SL (plus the sink prefix) is kept in EVERY layer's cache with one index list.  A
+    numpy mirror is advanced with the oracle's select / compact from the same fp32 scores; the
+    caches and SL must stay bit-identical, the scores within tolerance of the oracle's."""
+    rng = np.random.default_rng(31)
+    N, D, n_layers, chunk, cap, n_sink = 2, 128, 3, 96, 320, 32
+    dm = N * D
+    bits = lambda shape, sc=1.0: wl.f32_to_bf16_bits((rng.standard_normal(shape) * sc).astype(np.float32))
+    w1, b1 = bits((64, 3 * dm), (3 * dm) ** -0.5), bits((64,), 0.3)
+    w2, b2 = bits((12, 64), 64 ** -0.5), bits((12,), 0.3)
+    dw = [to_device_bf16(a) for a in (w1, b1, w2, b2)]
+    head = pafu.Head(dw[0], dw[1], dw[2], dw[3], wl.ACT_SILU, wl.FINAL_NONE)
+    ws = torch.zeros(pafu.pafu_workspace_bytes(pafu.Shape(N, D, [0, cap], [0, chunk]), None, head),
+                     dtype=torch.uint8, device="cuda")
+    K = [np.zeros((0, N, D), np.uint16) for _ in range(n_layers)]; V = [k.copy() for k in K]   # mirror
+    SL = np.zeros(0, np.float32)
+    dK = [to_device_bf16(k) for k in K]; dV = [to_device_bf16(v) for v in V]
+    dSL = torch.zeros(0, device="cuda")
+    pruned = 0
+    for c in range(7):
+        newK = [bits((chunk, N, D)) for _ in range(n_layers)]; newV = [bits((chunk, N, D)) for _ in range(n_layers)]
+        if c == 0:
+            first_K = newK
+        q = bits((chunk, N, D))
+        s_new = torch.full((chunk,), float("nan"), device="cuda")
+        pafu.pafu_score_qkv(head, to_device_bf16(q), to_device_bf16(newK[-1]), to_device_bf16(newV[-1]), s_new, ws,
+                            ld=dm)
+        X = np.concatenate([q.reshape(chunk, dm), newK[-1].reshape(chunk, dm), newV[-1].reshape(chunk, dm)], axis=1)
+        close(s_new.cpu().numpy(), oracle.score(np.ascontiguousarray(X), w1, b1, w2, b2, wl.ACT_SILU, wl.FINAL_NONE),
+              "chunk score")
+        T = SL.shape[0]
+        if T + chunk > cap:
+            budget = cap - chunk
+            shape = pafu.Shape(N, D, [0, T], None)
+            pol = pafu.make_policy(n_sink, 0, [budget], 1)
+            idx = torch.full((budget,), -1, dtype=torch.int32, device="cuda")
+            pafu.pafu_select(dSL, shape, pol, idx)
+            want_idx = oracle.select(SL, n_sink, 0, budget)
+            assert np.array_equal(idx.cpu().numpy(), want_idx)
+            Kc = [torch.zeros((budget, N, D), dtype=torch.bfloat16, device="cuda") for _ in range(n_layers)]
+            Vc = [torch.zeros_like(k) for k in Kc]
+            SLc = torch.zeros(budget, device="cuda")
+            pafu.pafu_compact_layers(dK, dV, dSL, idx, shape, pol, Kc, Vc, SLc)
+            K = [oracle.compact(k, want_idx) for k in K]; V = [oracle.compact(v, want_idx) for v in V]
+            SL = oracle.compact(SL, want_idx)
+            dK, dV, dSL = Kc, Vc, SLc
+            pruned += 1
+        # append the new chunk (its scores are the GPU's own fp32 values on both sides)
+        s_host = s_new.cpu().numpy()
+        K = [np.concatenate([a, b]) for a, b in zip(K, newK)]; V = [np.concatenate([a, b]) for a, b in zip(V, newV)]
+        SL = np.concatenate([SL, s_host])
+        dK = [torch.cat([a, to_device_bf16(b)]) for a, b in zip(dK, newK)]
+        dV = [torch.cat([a, to_device_bf16(b)]) for a, b in zip(dV, newV)]
+        dSL = torch.cat([dSL, s_new])
+        assert SL.shape[0] <= cap
+        for l in range(n_layers):
+            assert np.array_equal(bf16_to_bits(dK[l]), K[l]) and np.array_equal(bf16_to_bits(dV[l]), V[l]), (c, l)
+        assert np.array_equal(dSL.cpu().numpy(), SL)
+    # the sink prefix (first tokens of the first chunk) survives every pruning round in every layer
+    assert pruned >= 3
+    for l in range(n_layers):
+        assert np.array_equal(K[l][:n_sink], first_K[l][:n_sink])
+
+
 # --------------------------------------------------------------- attention through indices
 def test_indexed_attention_matches_oracle_and_compacted_path():
     """Select(KV; ids) applied inside the attention loader (Eq. 7's index set) instead of as a
