@@ -258,3 +258,68 @@ void pafu_oracle_sse(const uint16_t *Q, const uint16_t *K, int64_t L, int32_t N,
     }
     free(low); free(diag); free(up);
 }
+
+/* ------------------------------------------------------------- sse, sampled columns ---
+ * The same definition (Eq. 4, Eq. 5) evaluated for a list of key positions only, for sequences
+ * too long to hold P: per head, every row's log-sum-exp is computed first (one streaming pass
+ * over all L x L logits), then for each listed key j the column P[i, j] = exp(z_ij - lse_i) is
+ * walked over all queries i and split by the query's block into the three maxima.
+ * Outputs: s [n_cols], comp [3, n_cols] = low, diag, up (comp may be NULL).
+ */
+void pafu_oracle_sse_cols(const uint16_t *Q, const uint16_t *K, int64_t L, int32_t N, int32_t D,
+                          int64_t LB, double scale, const int64_t *cols, int64_t n_cols,
+                          double *s, double *comp) {
+    const int64_t dm = (int64_t)N * D;
+    double *low = (double *)calloc((size_t)n_cols, sizeof(double));
+    double *diag = (double *)calloc((size_t)n_cols, sizeof(double));
+    double *up = (double *)calloc((size_t)n_cols, sizeof(double));
+    double *q = (double *)malloc(sizeof(double) * (size_t)L * D);
+    double *k = (double *)malloc(sizeof(double) * (size_t)L * D);
+    double *lse = (double *)malloc(sizeof(double) * (size_t)L);
+    for (int32_t n = 0; n < N; ++n) {
+        for (int64_t i = 0; i < L; ++i)
+            for (int32_t d = 0; d < D; ++d) {
+                q[i * D + d] = bf16_to_f64(Q[i * dm + n * D + d]);
+                k[i * D + d] = bf16_to_f64(K[i * dm + n * D + d]);
+            }
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < L; ++i) {
+            double *z = (double *)malloc(sizeof(double) * (size_t)L);
+            double m = -INFINITY;
+            for (int64_t j = 0; j < L; ++j) {
+                double acc = 0.0;
+                for (int32_t d = 0; d < D; ++d) acc += q[i * D + d] * k[j * D + d];
+                z[j] = acc * scale;
+                if (z[j] > m) m = z[j];
+            }
+            double l = 0.0;
+            for (int64_t j = 0; j < L; ++j) l += exp(z[j] - m);
+            lse[i] = m + log(l);
+            free(z);
+        }
+#pragma omp parallel for schedule(static)
+        for (int64_t c = 0; c < n_cols; ++c) {
+            const int64_t j = cols[c];
+            double mlow = 0.0, mdiag = 0.0, mup = 0.0;
+            for (int64_t i = 0; i < L; ++i) {
+                double acc = 0.0;
+                for (int32_t d = 0; d < D; ++d) acc += q[i * D + d] * k[j * D + d];
+                const double p = exp(acc * scale - lse[i]);
+                const int64_t lo = (i / LB) * LB, hi = lo + LB;
+                if (j < lo) { if (p > mlow) mlow = p; }
+                else if (j < hi) { if (p > mdiag) mdiag = p; }
+                else { if (p > mup) mup = p; }
+            }
+            low[c] += mlow; diag[c] += mdiag; up[c] += mup;
+        }
+    }
+    for (int64_t c = 0; c < n_cols; ++c) {
+        const int64_t j = cols[c];
+        low[c] /= N; diag[c] /= N; up[c] /= N;
+        if (j < LB) s[c] = (diag[c] + low[c]) / 2.0;
+        else if (j < L - LB) s[c] = (up[c] + diag[c] + low[c]) / 3.0;
+        else s[c] = (diag[c] + up[c]) / 2.0;
+        if (comp) { comp[c] = low[c]; comp[n_cols + c] = diag[c]; comp[2 * n_cols + c] = up[c]; }
+    }
+    free(low); free(diag); free(up); free(q); free(k); free(lse);
+}

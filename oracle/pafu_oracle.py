@@ -61,6 +61,10 @@ def _load():
         lib.pafu_oracle_sse.argtypes = [_c_u16p, _c_u16p, ctypes.c_int64, ctypes.c_int32,
                                         ctypes.c_int32, ctypes.c_int64, ctypes.c_double, _c_f64p,
                                         _c_f64p]
+        lib.pafu_oracle_sse_cols.restype = None
+        lib.pafu_oracle_sse_cols.argtypes = [_c_u16p, _c_u16p, ctypes.c_int64, ctypes.c_int32,
+                                             ctypes.c_int32, ctypes.c_int64, ctypes.c_double, _c_i64p,
+                                             ctypes.c_int64, _c_f64p, _c_f64p]
         _lib = lib
     return _lib
 
@@ -164,4 +168,20 @@ def sse(Q: np.ndarray, K: np.ndarray, block_len: int, scale: Optional[float] = N
     comp = np.empty((3, L), dtype=np.float64)
     _load().pafu_oracle_sse(_p(Q, _c_u16p), _p(K, _c_u16p), L, N, D, block_len, float(scale),
                             _p(s, _c_f64p), _p(comp, _c_f64p))
+    return s, comp
+
+
+def sse_cols(Q: np.ndarray, K: np.ndarray, block_len: int, cols: Sequence[int],
+             scale: Optional[float] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Eq. 4 / Eq. 5 for the listed key positions only (no L x L matrix is held): returns
+    (s [n_cols], comp [3, n_cols])."""
+    Q = _u16(Q); K = _u16(K)
+    L, N, D = Q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    c = np.ascontiguousarray(cols, dtype=np.int64)
+    s = np.empty(c.shape[0], dtype=np.float64)
+    comp = np.empty((3, c.shape[0]), dtype=np.float64)
+    _load().pafu_oracle_sse_cols(_p(Q, _c_u16p), _p(K, _c_u16p), L, N, D, block_len, float(scale),
+                                 _p(c, _c_i64p), c.shape[0], _p(s, _c_f64p), _p(comp, _c_f64p))
     return s, comp

@@ -379,6 +379,27 @@ def test_sse_matches_oracle(L, N, LB):
     assert torch.equal(s, s2)
 
 
+def test_sse_full_size_sampled_columns():
+    """The paper's training length (21 frames x 1560 tokens, blocks of 4680; Appendix A), one head:
+    a seeded sample of key positions, block and tile boundaries included, against the oracle."""
+    L, N, D, LB = 32760, 1, 128, 4680
+    rng = np.random.default_rng(3)
+    Q = wl.f32_to_bf16_bits((rng.standard_normal((L, N, D)) * 1.5).astype(np.float32))
+    K = wl.f32_to_bf16_bits((rng.standard_normal((L, N, D)) * 1.5).astype(np.float32))
+    cols = sorted(set([0, 127, 128, LB - 1, LB, LB + 1, 4607, 4608, 2 * LB - 1, 2 * LB, L - LB - 1, L - LB, L - 1])
+                  | set(rng.choice(L, size=19, replace=False).tolist()))
+    want_s, want_c = oracle.sse_cols(Q, K, LB, cols)
+    ws = torch.zeros(pafu.pafu_sse_workspace_bytes(L, N, D, LB), dtype=torch.uint8, device="cuda")
+    s = torch.full((L,), float("nan"), device="cuda"); comp = torch.full((3, L), float("nan"), device="cuda")
+    pafu.pafu_sse(to_device_bf16(Q), to_device_bf16(K), None, LB, 0.0, s, comp, ws)
+    assert pafu.pafu_workspace_status(ws) == 0
+    got_s, got_c = s.cpu().numpy(), comp.cpu().numpy()
+    assert np.all(np.isfinite(got_s)) and np.all(got_c >= 0) and np.all(got_c <= 1.0 + 1e-5)
+    assert np.all(got_c[2, :LB] == 0) and np.all(got_c[0, L - LB:] == 0)     # classes without queries
+    assert np.allclose(got_c[:, cols], want_c, rtol=1e-3, atol=1e-7), np.abs(got_c[:, cols] - want_c).max()
+    assert np.allclose(got_s[cols], want_s, rtol=1e-3, atol=1e-7)
+
+
 # ---------------------------------------------------------------------------------- step
 @pytest.mark.parametrize("w", SMALL, ids=lambda w: "%s-d%d" % (w.name, w.d_head))
 def test_step_equals_four_calls_and_oracle(w):

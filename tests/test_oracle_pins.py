@@ -372,3 +372,22 @@ def test_sse_brute_force_index_sets():
         w = (want[1, j] + want[0, j]) / 2 if j < LB else ((want[2, j] + want[1, j] + want[0, j]) / 3 if j < L - LB
                                                             else (want[1, j] + want[2, j]) / 2)
         assert abs(s[j] - w) < 1e-14
+
+
+def test_sse_sampled_columns_equal_full_and_dense():
+    # the streaming variant used at full size: same numbers as the full oracle, and as dense torch
+    rng = np.random.default_rng(8)
+    L, N, D, LB = 37, 2, 8, 9
+    Q = bf(rng.standard_normal((L, N, D)).astype(np.float32) * 2)
+    K = bf(rng.standard_normal((L, N, D)).astype(np.float32) * 2)
+    cols = [0, 8, 9, 17, 18, 27, 28, 35, 36]
+    s, comp = oracle.sse(Q, K, LB)
+    s2, comp2 = oracle.sse_cols(Q, K, LB, cols)
+    assert np.allclose(s2, s[cols], atol=1e-14) and np.allclose(comp2, comp[:, cols], atol=1e-14)
+    tq = torch.from_numpy(f32(Q)).double(); tk = torch.from_numpy(f32(K)).double()
+    P = torch.softmax(torch.einsum("qnd,knd->nqk", tq, tk) / math.sqrt(D), dim=-1).numpy()
+    for ci, j in enumerate(cols):
+        qb = np.arange(L) // LB
+        for cls, mask in enumerate((qb > j // LB, qb == j // LB, qb < j // LB)):
+            want = np.mean([P[n, mask, j].max() if mask.any() else 0.0 for n in range(N)])
+            assert abs(comp2[cls, ci] - want) < 1e-13
