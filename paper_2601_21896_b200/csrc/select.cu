@@ -3,7 +3,7 @@
 // ascending token indices, ties to the lower index.
 //
 // The step moves a few hundred KB, so it is latency-bound: a cluster of eight CTAs per stream
-// with the candidates in registers (streams up to 32768 candidates), one CTA re-reading L2
+// with the candidates in registers (streams up to 131072 candidates), one CTA re-reading L2
 // for longer streams.
 //   1. fp32 scores map to order-preserving 32-bit keys (-0 folded onto +0, NaN lowest).
 //   2. MSB-first radix select (4 passes of 8 bits, shared-memory histograms) finds the key of
@@ -55,20 +55,26 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
 }
 
 constexpr int kSelCluster = 8;                        // CTAs cooperating on one stream
-constexpr int kSelRows = 4;                           // candidates per thread held in registers
-constexpr int kSelPerCta = kSelRows * kSelThreads;    // 4096
-constexpr int kSelRegCap = kSelCluster * kSelPerCta;  // 32768 candidates
+constexpr int kSelRowsSmall = 4, kSelRowsLarge = 16;  // candidates per thread held in registers
+constexpr int kSelCapSmall = kSelCluster * kSelRowsSmall * kSelThreads;   // 32768 candidates
+constexpr int kSelRegCap = kSelCluster * kSelRowsLarge * kSelThreads;     // 131072 candidates
 
 // Streams with at most kSelRegCap candidates: a cluster of eight CTAs per stream.  Candidate j
-// lives in CTA j / 4096, row (j / 1024) % 4, thread j % 1024, loaded once and kept in registers.
+// lives in CTA j / (ROWS * 1024), row (j / 1024) % ROWS, thread j % 1024, loaded once and kept in
+// registers; ROWS = 4 serves streams up to 32768 candidates, ROWS = 16 those up to 131072 (a
+// 93 600-token cache), each stream by exactly one of the two instantiations.
 // Every radix pass (12 + 10 + 10 bits) builds one shared-memory histogram per CTA; CTA r then
 // sums slice r of the bins over all eight histograms through distributed shared memory, the
 // slice totals are exchanged, and the CTA whose slice holds the k-th largest key finds the bin
 // and tells the others.  Emission: warp ballots per row, one block scan over the 4 x 32
 // (row, warp) counts, and the CTA totals exchanged through distributed shared memory give every
 // kept candidate its ascending output slot.
+template <int kSelRows>
 __global__ void __launch_bounds__(kSelThreads)
 select_cluster_kernel(const float* __restrict__ scores, StreamTable st, int32_t* __restrict__ idx) {
+    constexpr int kSelPerCta = kSelRows * kSelThreads;
+    constexpr int kCap = kSelCluster * kSelPerCta;
+    constexpr int kCapBelow = kSelRows == kSelRowsSmall ? 0 : kSelCapSmall;    // smaller streams: the other instantiation
     grid_dep_wait();
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
@@ -92,7 +98,7 @@ select_cluster_kernel(const float* __restrict__ scores, StreamTable st, int32_t*
     const int ns = (int)st.n_sink[s], nr = (int)st.n_recent[s];
     const int k = (int)st.k[s];
     const int c0 = ns, M = T - nr - ns;
-    if (M > kSelRegCap) return;                           // the streaming kernel owns this stream
+    if (M > kCap || M <= kCapBelow) return;               // another kernel owns this stream
     const float* sc = scores + st.cu_T[s] + c0;
     int32_t* out = idx + st.cu_B[s];
     const int j0 = rank * kSelPerCta;
@@ -356,18 +362,23 @@ pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* i
                           cudaStream_t stream) {
     if (st.n_streams == 0 || st.cu_B[st.n_streams] == 0) return PAFU_OK;
     // both kernels run over all streams; each stream is handled by exactly one of them
-    bool any_regs = false, any_stream = false;
+    bool any_small = false, any_large = false, any_stream = false;
     for (int s = 0; s < st.n_streams; ++s) {
         const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
-        const bool regs = B < T && T - st.n_sink[s] - st.n_recent[s] <= kSelRegCap;
-        any_regs |= regs;
+        const int64_t M = T - st.n_sink[s] - st.n_recent[s];
+        const bool regs = B < T && M <= kSelRegCap;
+        any_small |= regs && M <= kSelCapSmall;
+        any_large |= regs && M > kSelCapSmall;
         any_stream |= !regs;
     }
-    if (any_regs) {
-        if (launch_dependent(select_cluster_kernel, dim3((unsigned)(st.n_streams * kSelCluster)), dim3(kSelThreads), 0,
-                             stream, kSelCluster, scores, st, idx) != cudaSuccess)
-            return PAFU_ERR_CUDA;
-    }
+    if (any_small &&
+        launch_dependent(select_cluster_kernel<kSelRowsSmall>, dim3((unsigned)(st.n_streams * kSelCluster)), dim3(kSelThreads), 0,
+                         stream, kSelCluster, scores, st, idx) != cudaSuccess)
+        return PAFU_ERR_CUDA;
+    if (any_large &&
+        launch_dependent(select_cluster_kernel<kSelRowsLarge>, dim3((unsigned)(st.n_streams * kSelCluster)), dim3(kSelThreads), 0,
+                         stream, kSelCluster, scores, st, idx) != cudaSuccess)
+        return PAFU_ERR_CUDA;
     if (any_stream &&
         launch_dependent(select_stream_kernel, dim3((unsigned)st.n_streams), dim3(kSelThreads), 0, stream, 1, scores, st,
                          idx) != cudaSuccess)
