@@ -341,6 +341,40 @@ def run_ours(args):
                    "value": world * n_layers * work["attn_flops"] / (idx_ms * 1e-3) / 1e12, "unit": UNIT,
                    "attn_ms": ia_ms, "attn_TFLOP/s": work["attn_flops"] / (ia_ms * 1e-3) / 1e12}
 
+    # ---- the same steps replayed from a CUDA graph (one graph = one pass over the buffer sets, or
+    # the n_layers of a denoising step): what is left of the host's launch work
+    graph = None
+    if args.graph:
+        try:
+            n_cap = n_sets if n_layers <= 1 else n_layers
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                for i in range(n_cap):
+                    layers[i % n_sets].step()
+            side.synchronize()
+            cg = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(cg, stream=side):
+                for i in range(n_cap):
+                    layers[i % n_sets].step()
+            reps = max(1, (steps * n_layers) // n_cap)
+            for _ in range(2):
+                cg.replay()
+            g0, g1 = new_events(2)
+            torch.cuda.synchronize()
+            g0.record(stream)
+            for _ in range(reps):
+                cg.replay()
+            g1.record(stream)
+            torch.cuda.synchronize()
+            for L in layers:
+                L.check_status()
+            g_ms = sharding.max_over_ranks(g0.elapsed_time(g1) / (reps * n_cap) * n_layers, device="cuda")
+            graph = {"ms_per_step": g_ms, "value": world * n_layers * work["attn_flops"] / (g_ms * 1e-3) / 1e12,
+                     "unit": UNIT, "steps_per_graph": n_cap / n_layers, "kernels_per_graph": n_cap * launches_per_step(w)}
+        except Exception as exc:      # capture is an optional extra: report, do not fail the run
+            graph = {"error": "%s: %s" % (type(exc).__name__, exc)}
+
     # ---- e2e: host buffers through pafu_step_host (H2D of inputs + D2H of results timed)
     L0 = layers[0]
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
@@ -502,6 +536,7 @@ def run_ours(args):
         },
         "score_qkv": qkv,
         "step_indexed": indexed,
+        "cuda_graph": graph,
         "sse": sse,
         "shared_index_compaction": shared,
         "layers_per_step": n_layers,
@@ -532,6 +567,8 @@ def main():
                          "denoising step of the 30-layer sweep (every layer has its own cache and head)")
     ap.add_argument("--shared-layers", type=int, default=30,
                     help="layers pruned with one shared index list in the shared-index timing; 0 skips it")
+    ap.add_argument("--graph", action=argparse.BooleanOptionalAction, default=True,
+                    help="also time the steps replayed from a captured CUDA graph")
     ap.add_argument("--sse-tokens", type=int, default=32760,
                     help="sequence length of the teacher-salience (Eq. 4/5) timing; 0 skips it")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

@@ -323,3 +323,36 @@ void pafu_oracle_sse_cols(const uint16_t *Q, const uint16_t *K, int64_t L, int32
     }
     free(low); free(diag); free(up); free(q); free(k); free(lse);
 }
+
+/* ------------------------------------------------------- global max pooling ---
+ * The "Max" alternative of the paper's ablation on the salience score (Sec. 4.3, Table 3):
+ * g_j = mean over heads of max over ALL queries i of P[n, i, j], P = softmax(Q K^T * scale).
+ */
+void pafu_oracle_sse_gmax(const uint16_t *Q, const uint16_t *K, int64_t L, int32_t N, int32_t D,
+                          double scale, double *g) {
+    const int64_t dm = (int64_t)N * D;
+    for (int64_t j = 0; j < L; ++j) g[j] = 0.0;
+    double *P = (double *)malloc(sizeof(double) * (size_t)L * (size_t)L);
+    for (int32_t n = 0; n < N; ++n) {
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < L; ++i) {
+            double *p = P + i * L;
+            double m = -INFINITY, l = 0.0;
+            for (int64_t j = 0; j < L; ++j) {
+                double acc = 0.0;
+                for (int32_t d = 0; d < D; ++d)
+                    acc += bf16_to_f64(Q[i * dm + n * D + d]) * bf16_to_f64(K[j * dm + n * D + d]);
+                p[j] = acc * scale;
+                if (p[j] > m) m = p[j];
+            }
+            for (int64_t j = 0; j < L; ++j) { p[j] = exp(p[j] - m); l += p[j]; }
+            for (int64_t j = 0; j < L; ++j) p[j] /= l;
+        }
+        for (int64_t j = 0; j < L; ++j) {
+            double mx = 0.0;
+            for (int64_t i = 0; i < L; ++i) if (P[i * L + j] > mx) mx = P[i * L + j];
+            g[j] += mx / N;
+        }
+    }
+    free(P);
+}

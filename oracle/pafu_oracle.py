@@ -61,6 +61,9 @@ def _load():
         lib.pafu_oracle_sse.argtypes = [_c_u16p, _c_u16p, ctypes.c_int64, ctypes.c_int32,
                                         ctypes.c_int32, ctypes.c_int64, ctypes.c_double, _c_f64p,
                                         _c_f64p]
+        lib.pafu_oracle_sse_gmax.restype = None
+        lib.pafu_oracle_sse_gmax.argtypes = [_c_u16p, _c_u16p, ctypes.c_int64, ctypes.c_int32,
+                                             ctypes.c_int32, ctypes.c_double, _c_f64p]
         lib.pafu_oracle_sse_cols.restype = None
         lib.pafu_oracle_sse_cols.argtypes = [_c_u16p, _c_u16p, ctypes.c_int64, ctypes.c_int32,
                                              ctypes.c_int32, ctypes.c_int64, ctypes.c_double, _c_i64p,
@@ -185,3 +188,14 @@ def sse_cols(Q: np.ndarray, K: np.ndarray, block_len: int, cols: Sequence[int],
     _load().pafu_oracle_sse_cols(_p(Q, _c_u16p), _p(K, _c_u16p), L, N, D, block_len, float(scale),
                                  _p(c, _c_i64p), c.shape[0], _p(s, _c_f64p), _p(comp, _c_f64p))
     return s, comp
+
+
+def sse_global_max(Q: np.ndarray, K: np.ndarray, scale: Optional[float] = None) -> np.ndarray:
+    """Global max pooling of the attention weights (the "Max" ablation, Sec. 4.3): [L]."""
+    Q = _u16(Q); K = _u16(K)
+    L, N, D = Q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    g = np.empty(L, dtype=np.float64)
+    _load().pafu_oracle_sse_gmax(_p(Q, _c_u16p), _p(K, _c_u16p), L, N, D, float(scale), _p(g, _c_f64p))
+    return g

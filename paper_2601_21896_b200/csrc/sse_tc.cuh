@@ -358,7 +358,7 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
 }
 
 // exp2 of the per-head maxima, mean over heads (head order), Eq. 5.
-__global__ void sse_finish_kernel(Params p, float* __restrict__ s, float* __restrict__ comp) {
+__global__ void sse_finish_kernel(Params p, float* __restrict__ s, float* __restrict__ comp, float* __restrict__ gmax) {
     grid_dep_wait();
     for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < p.L; j += (int64_t)gridDim.x * blockDim.x) {
         float c[3];
@@ -374,6 +374,14 @@ __global__ void sse_finish_kernel(Params p, float* __restrict__ s, float* __rest
         else v = (c[1] + c[2]) * 0.5f;
         s[j] = v;
         if (comp != nullptr) { comp[j] = c[0]; comp[p.L + j] = c[1]; comp[2 * p.L + j] = c[2]; }
+        if (gmax != nullptr) {          // max over all queries per head, then the mean over heads
+            float acc = 0.f;
+            for (int n = 0; n < p.n_heads; ++n) {
+                const float* m = p.M + (int64_t)n * 3 * p.L + j;
+                acc += exp2f(fmaxf(fmaxf(m[0], m[p.L]), m[2 * p.L]));
+            }
+            gmax[j] = acc / (float)p.n_heads;
+        }
     }
 }
 
@@ -398,7 +406,7 @@ inline size_t aug_bytes(const Params& p) { return (size_t)p.n_heads * p.n_qt * k
 inline size_t maxima_bytes(const Params& p) { return (size_t)p.n_heads * 3 * p.L * 4; }
 
 inline pafu_status launch(const uint16_t* Q, const uint16_t* K, const float* lse, int64_t L, int64_t LB,
-                          int n_heads, float scale, float* s, float* comp, uint16_t* q_aug, float* M,
+                          int n_heads, float scale, float* s, float* comp, float* gmax, uint16_t* q_aug, float* M,
                           int* status, cudaStream_t stream) {
     Params p = make_params(L, LB, n_heads, scale);
     p.q_aug = q_aug; p.M = M; p.status = status;
@@ -421,7 +429,7 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* K, const float* lse
     if (launch_dependent(sse_tc_kernel, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mK, p, n_items) != cudaSuccess)
         return PAFU_ERR_CUDA;
     const int g2 = (int)((L + 255) / 256 < 4 * sms ? (L + 255) / 256 : 4 * sms);
-    if (launch_dependent(sse_finish_kernel, dim3(g2), dim3(256), 0, stream, 1, p, s, comp) != cudaSuccess)
+    if (launch_dependent(sse_finish_kernel, dim3(g2), dim3(256), 0, stream, 1, p, s, comp, gmax) != cudaSuccess)
         return PAFU_ERR_CUDA;
     return PAFU_OK;
 }

@@ -391,3 +391,17 @@ def test_sse_sampled_columns_equal_full_and_dense():
         for cls, mask in enumerate((qb > j // LB, qb == j // LB, qb < j // LB)):
             want = np.mean([P[n, mask, j].max() if mask.any() else 0.0 for n in range(N)])
             assert abs(comp2[cls, ci] - want) < 1e-13
+
+
+def test_sse_global_max_against_dense_torch():
+    rng = np.random.default_rng(12)
+    L, N, D = 19, 3, 8
+    Q = bf(rng.standard_normal((L, N, D)).astype(np.float32) * 2)
+    K = bf(rng.standard_normal((L, N, D)).astype(np.float32) * 2)
+    g = oracle.sse_global_max(Q, K)
+    tq = torch.from_numpy(f32(Q)).double(); tk = torch.from_numpy(f32(K)).double()
+    P = torch.softmax(torch.einsum("qnd,knd->nqk", tq, tk) / math.sqrt(D), dim=-1)
+    assert np.allclose(g, P.max(dim=1).values.mean(dim=0).numpy(), atol=1e-14)
+    # it dominates each of the three block-wise components and equals their maximum for one head
+    _, comp = oracle.sse(Q[:, :1], K[:, :1], 5)
+    assert np.allclose(oracle.sse_global_max(Q[:, :1], K[:, :1]), comp.max(axis=0), atol=1e-14)
