@@ -100,6 +100,44 @@ def test_argument_errors_are_caught_on_the_host(L):
     assert L.pafu_workspace_bytes(ctypes.byref(sh.c), pol, None) % 256 == 0
 
 
+def test_newer_entry_points_reject_bad_arguments_on_host(L):
+    fake = 0x7f0000000000
+    sh = pafu.Shape(2, 128, [0, 512], [0, 64])
+    sh64 = pafu.Shape(2, 64, [0, 512], [0, 64])
+    pol = pafu.make_policy(4, 64, 128, 1)
+    cu_B = np.array([0, 128], dtype=np.int64)
+    # attention through indices: d_head 128 only, idx required, retained count cannot exceed the cache
+    call = lambda shape, idx, cb: L.pafu_chunk_attn_indexed(fake, fake, fake, idx, cb.ctypes.data, fake, fake,
+                                                            ctypes.byref(shape.c), 0.0, fake, None, fake, 1 << 30, None)
+    assert call(sh64, fake, cu_B) == 3
+    assert call(sh, None, cu_B) == 1
+    assert call(sh, fake, np.array([0, 513], dtype=np.int64)) == 1
+    assert call(sh, fake + 4, cu_B) == 5
+    assert L.pafu_step_indexed(None, None) == 1
+    # all-layer compaction: pointer arrays, layer count
+    arr = (ctypes.c_void_p * 2)(fake, fake + 4096)
+    out = (ctypes.c_void_p * 2)(fake + 8192, fake + 12288)
+    cl = lambda K, n, Kc: L.pafu_compact_layers(K, arr, n, None, fake, ctypes.byref(sh.c), pol, Kc, out, None, None)
+    assert cl(arr, -1, out) == 1
+    assert cl(arr, 65, out) == 3
+    assert cl(None, 2, out) == 1
+    assert cl(arr, 2, arr) == 1                                     # in place
+    assert cl((ctypes.c_void_p * 2)(fake, None), 2, out) == 1       # a missing layer
+    assert cl(arr, 0, out) == 0                                     # no layers: no-op
+    # teacher salience target
+    sse = lambda Lt, N, D, LB, scale, s, ws, nb: L.pafu_sse(fake, fake, None, Lt, N, D, LB, scale, s, None, None, ws, nb, None)
+    need = L.pafu_sse_workspace_bytes(1000, 2, 128, 256)
+    assert need > 0 and need % 256 == 0
+    assert L.pafu_sse_workspace_bytes(1000, 2, 64, 256) == 0 and L.pafu_sse_workspace_bytes(0, 2, 128, 256) == 0
+    assert sse(1000, 2, 64, 256, 0.0, fake, fake, need) == 3
+    assert sse(0, 2, 128, 256, 0.0, fake, fake, need) == 1
+    assert sse(1000, 2, 128, 0, 0.0, fake, fake, need) == 1
+    assert sse(1000, 2, 128, 256, -1.0, fake, fake, need) == 1
+    assert sse(1000, 2, 128, 256, 0.0, None, fake, need) == 1
+    assert sse(1000, 2, 128, 256, 0.0, fake, fake + 16, need) == 5
+    assert sse(1000, 2, 128, 256, 0.0, fake, fake, need - 1) == 4
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
