@@ -120,11 +120,11 @@ __host__ __device__ inline int64_t total_cost(const StreamTable& st, int n_heads
 // can start inside an item (t0 > 0) and only its last run can stop inside one (t1 < nt).
 struct SegIter {
     int64_t cur, c1;
-    __device__ SegIter(const Params& p, int cta, int n_cta) {
+    __host__ __device__ SegIter(const Params& p, int cta, int n_cta) {
         cur = p.total_cost * cta / n_cta;
         c1 = p.total_cost * (cta + 1) / n_cta;
     }
-    __device__ bool next(const Params& p, Seg& g) {
+    __host__ __device__ bool next(const Params& p, Seg& g) {
         while (cur < c1) {
             int64_t c = cur;
             int s = 0;
@@ -667,82 +667,109 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     if (warp == 8) tmem_dealloc(tmem, 512);
 }
 
-// Merges the partials of every item that was split across CTAs.  Blocks 2b and 2b+1 own the
-// two slots of the item that CTA b of the main kernel began (its last run, stored as piece 1)
-// and add the following CTAs' continuation pieces (their first run, piece 0) in key order.
-// Each of the 32 warps handles four rows, so all loads of a block are in flight together.
+// Merges the partials of every item that was split across CTAs.  The host walks the CTAs'
+// shares once per launch and passes the work as a table: item i was begun by CTA cta[first]
+// (its last run, stored as that CTA's piece 1) and continued by the following entries (each
+// CTA's first run, piece 0), in key order, which keeps the result deterministic.  Eight blocks
+// of 256 threads per item (two slots x four groups of 32 rows); a warp handles four rows, so
+// all loads of a block are in flight together.
 constexpr int kMergeRows = 4;
-__global__ void __launch_bounds__(1024)
-attn_tc_merge_kernel(const __grid_constant__ Params p, int n_cta) {
+constexpr int kMergeThreads = 256;
+constexpr int kMergeBlocksPerItem = 2 * (kBM / (kMergeThreads / 32 * kMergeRows));   // 8
+struct MergeItem {
+    int32_t o_row;        // row of O (and LSE column) of the item's first query
+    int32_t rows;         // valid query rows of the item (<= 256)
+    int16_t head, n_slots;
+    int16_t first, n_pieces;   // entries [first, first + n_pieces) of MergeTable::cta
+};
+struct MergeTable {
+    int32_t n_items;
+    MergeItem item[kMaxGrid];
+    int16_t cta[2 * kMaxGrid];
+};
+
+__global__ void __launch_bounds__(kMergeThreads)
+attn_tc_merge_kernel(const __grid_constant__ MergeTable tb, const float* __restrict__ pieces, float scale,
+                     int n_heads, int64_t total_Lq, uint16_t* __restrict__ O, float* __restrict__ LSE) {
     grid_dep_wait();
-    __shared__ int piece_cta[kMaxGrid];
-    __shared__ int n_pieces_sh;
-    const int b = blockIdx.x >> 1, slot = blockIdx.x & 1;
-    Seg g, last;
-    bool have = false;
-    {
-        SegIter iter(p, b, n_cta);
-        while (iter.next(p, g)) { last = g; have = true; }
+    const MergeItem& it = tb.item[blockIdx.x / kMergeBlocksPerItem];
+    const int slot = (blockIdx.x / (kMergeBlocksPerItem / 2)) & 1;
+    const int group = blockIdx.x % (kMergeBlocksPerItem / 2);
+    if (slot >= it.n_slots) return;                                    // block-uniform
+    const int n_pieces = it.n_pieces;
+    const float sl2 = scale * 1.4426950408889634f;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;        // 32 float4 per row
+    const int r0 = group * (kMergeThreads / 32 * kMergeRows) + warp * kMergeRows;
+    float M[kMergeRows], L[kMergeRows];
+    float4 acc[kMergeRows];
+#pragma unroll
+    for (int q = 0; q < kMergeRows; ++q) { M[q] = -INFINITY; L[q] = 0.f; acc[q] = make_float4(0.f, 0.f, 0.f, 0.f); }
+    for (int i = 0; i < n_pieces; ++i) {
+        const float* piece = pieces + ((size_t)tb.cta[it.first + i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
+#pragma unroll
+        for (int q = 0; q < kMergeRows; ++q) M[q] = fmaxf(M[q], piece[2 * kBM * kD + slot * kBM + r0 + q]);
     }
-    if (!have || last.piece != 1 || slot >= last.n_slots) return;      // block-uniform
-    if (threadIdx.x == 0) {
-        int n = 0, t = last.t1;
-        piece_cta[n++] = b;
+    for (int i = 0; i < n_pieces; ++i) {
+        const float* piece = pieces + ((size_t)tb.cta[it.first + i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
+        float w[kMergeRows], l[kMergeRows];
+        float4 v[kMergeRows];
+#pragma unroll
+        for (int q = 0; q < kMergeRows; ++q) {
+            const int r = slot * kBM + r0 + q;
+            w[q] = piece[2 * kBM * kD + r];
+            l[q] = piece[2 * kBM * kD + 2 * kBM + r];
+            v[q] = reinterpret_cast<const float4*>(piece + (size_t)r * kD)[lane];
+        }
+#pragma unroll
+        for (int q = 0; q < kMergeRows; ++q) {
+            const float ww = fast_exp2((w[q] - M[q]) * sl2);
+            L[q] += ww * l[q];
+            acc[q].x += ww * v[q].x; acc[q].y += ww * v[q].y; acc[q].z += ww * v[q].z; acc[q].w += ww * v[q].w;
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < kMergeRows; ++q) {
+        const int row = slot * kBM + r0 + q;
+        if (row >= it.rows) continue;
+        const float inv = (L[q] > 0.f) ? 1.0f / L[q] : 0.f;
+        uint16_t* dst = O + (((int64_t)it.o_row + row) * n_heads + it.head) * kD + lane * 4;
+        uint2 o;
+        o.x = pack_bf16(acc[q].x * inv, acc[q].y * inv);
+        o.y = pack_bf16(acc[q].z * inv, acc[q].w * inv);
+        *reinterpret_cast<uint2*>(dst) = o;
+        if (LSE != nullptr && lane == 0)
+            LSE[(int64_t)it.head * total_Lq + it.o_row + row] = (L[q] > 0.f) ? M[q] * scale + logf(L[q]) : -INFINITY;
+    }
+}
+
+// Host side of the merge: which CTAs hold the pieces of which item.
+inline void build_merge_table(const Params& p, int n_cta, MergeTable& tb) {
+    tb.n_items = 0;
+    int n_list = 0;
+    Seg g, last;
+    for (int b = 0; b < n_cta; ++b) {
+        bool have = false;
+        {
+            SegIter iter(p, b, n_cta);
+            while (iter.next(p, g)) { last = g; have = true; }
+        }
+        if (!have || last.piece != 1) continue;
+        MergeItem& it = tb.item[tb.n_items++];
+        it.o_row = (int32_t)(p.st.cu_Lq[last.stream] + last.q0);
+        const int64_t left = last.Lq - last.q0;
+        it.rows = (int32_t)(left < 2 * kBM ? left : 2 * kBM);
+        it.head = (int16_t)last.head;
+        it.n_slots = (int16_t)last.n_slots;
+        it.first = (int16_t)n_list;
+        tb.cta[n_list++] = (int16_t)b;
+        int t = last.t1;
         for (int c = b + 1; c < n_cta && t < last.nt; ++c) {
             SegIter iter(p, c, n_cta);
             if (!iter.next(p, g)) continue;    // an empty share holds no piece
             t = g.t1;
-            piece_cta[n++] = c;
+            tb.cta[n_list++] = (int16_t)c;
         }
-        n_pieces_sh = n;
-    }
-    __syncthreads();
-    const int n_pieces = n_pieces_sh;
-    const float sl2 = p.scale * 1.4426950408889634f;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;   // 32 float4 per row
-    const float* __restrict__ pieces = p.pieces;
-    for (int r0 = warp * kMergeRows; r0 < kBM; r0 += 32 * kMergeRows) {   // one pass with 32 warps
-        float M[kMergeRows], L[kMergeRows];
-        float4 acc[kMergeRows];
-#pragma unroll
-        for (int q = 0; q < kMergeRows; ++q) { M[q] = -INFINITY; L[q] = 0.f; acc[q] = make_float4(0.f, 0.f, 0.f, 0.f); }
-        for (int i = 0; i < n_pieces; ++i) {
-            const float* piece = pieces + ((size_t)piece_cta[i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
-#pragma unroll
-            for (int q = 0; q < kMergeRows; ++q) M[q] = fmaxf(M[q], piece[2 * kBM * kD + slot * kBM + r0 + q]);
-        }
-        for (int i = 0; i < n_pieces; ++i) {
-            const float* piece = pieces + ((size_t)piece_cta[i] * 2 + (i == 0 ? 1 : 0)) * kPieceFloats;
-            float w[kMergeRows], l[kMergeRows];
-            float4 v[kMergeRows];
-#pragma unroll
-            for (int q = 0; q < kMergeRows; ++q) {
-                const int r = slot * kBM + r0 + q;
-                w[q] = piece[2 * kBM * kD + r];
-                l[q] = piece[2 * kBM * kD + 2 * kBM + r];
-                v[q] = reinterpret_cast<const float4*>(piece + (size_t)r * kD)[lane];
-            }
-#pragma unroll
-            for (int q = 0; q < kMergeRows; ++q) {
-                const float ww = fast_exp2((w[q] - M[q]) * sl2);
-                L[q] += ww * l[q];
-                acc[q].x += ww * v[q].x; acc[q].y += ww * v[q].y; acc[q].z += ww * v[q].z; acc[q].w += ww * v[q].w;
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < kMergeRows; ++q) {
-            const int64_t row = last.q0 + slot * kBM + r0 + q;
-            if (row >= last.Lq) continue;
-            const float inv = (L[q] > 0.f) ? 1.0f / L[q] : 0.f;
-            uint16_t* dst = p.O + ((p.st.cu_Lq[last.stream] + row) * p.n_heads + last.head) * kD + lane * 4;
-            uint2 o;
-            o.x = pack_bf16(acc[q].x * inv, acc[q].y * inv);
-            o.y = pack_bf16(acc[q].z * inv, acc[q].w * inv);
-            *reinterpret_cast<uint2*>(dst) = o;
-            if (p.LSE != nullptr && lane == 0)
-                p.LSE[(int64_t)last.head * p.total_Lq + p.st.cu_Lq[last.stream] + row] =
-                    (L[q] > 0.f) ? M[q] * p.scale + logf(L[q]) : -INFINITY;
-        }
+        it.n_pieces = (int16_t)(n_list - it.first);
     }
 }
 
@@ -808,7 +835,11 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
                 : launch_dependent(attn_tc_kernel<false>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mKc, mVc, mKq, mVq, p)) != cudaSuccess)
         return PAFU_ERR_CUDA;
     if (grid > 1) {
-        if (launch_dependent(attn_tc_merge_kernel, dim3(2 * grid), dim3(1024), 0, stream, 1, p, grid) != cudaSuccess)
+        MergeTable tb;
+        build_merge_table(p, grid, tb);
+        if (tb.n_items > 0 &&
+            launch_dependent(attn_tc_merge_kernel, dim3(tb.n_items * kMergeBlocksPerItem), dim3(kMergeThreads), 0, stream, 1,
+                             tb, (const float*)pieces, scale, (int)n_heads, nQ, O, LSE) != cudaSuccess)
             return PAFU_ERR_CUDA;
     }
     return PAFU_OK;
