@@ -314,6 +314,9 @@ pafu_status pafu_step_host(const pafu_step_args* args, void* arena, size_t arena
  *   comp      device fp32 [3, L], out: low, diag, up; or NULL
  *   gmax      device fp32 [L], out, or NULL: mean over heads of max_i P[n,i,j] over ALL queries -
  *             global max pooling, the "Max" alternative of the paper's ablation (Sec. 4.3, Table 3)
+ *   gavg      device fp32 [L], out, or NULL: mean over heads and over ALL queries of P[n,i,j] -
+ *             global average pooling, the "Avg" alternative of the same ablation; asking for it
+ *             costs one exponential per (query, key, head) on top of the contraction
  *   ws        device workspace of pafu_sse_workspace_bytes(...), 256-byte aligned, status header
  *             (first 256 bytes) zeroed by the caller; read it back with pafu_workspace_status
  * Supported: d_head = 128, L < 2^31.  fp32 accumulation; results agree with the definition to
@@ -321,7 +324,7 @@ pafu_status pafu_step_host(const pafu_step_args* args, void* arena, size_t arena
 size_t pafu_sse_workspace_bytes(int64_t L, int32_t n_heads, int32_t d_head, int64_t block_len);
 pafu_status pafu_sse(const uint16_t* Q, const uint16_t* K, const float* LSE, int64_t L,
                      int32_t n_heads, int32_t d_head, int64_t block_len, float scale,
-                     float* s, float* comp, float* gmax, void* ws, size_t ws_bytes, void* stream);
+                     float* s, float* comp, float* gmax, float* gavg, void* ws, size_t ws_bytes, void* stream);
 
 #ifdef __cplusplus
 }

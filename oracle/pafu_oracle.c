@@ -326,12 +326,13 @@ void pafu_oracle_sse_cols(const uint16_t *Q, const uint16_t *K, int64_t L, int32
 
 /* ------------------------------------------------------- global max pooling ---
  * The "Max" alternative of the paper's ablation on the salience score (Sec. 4.3, Table 3):
- * g_j = mean over heads of max over ALL queries i of P[n, i, j], P = softmax(Q K^T * scale).
+ * g_j = mean over heads of max over ALL queries i of P[n, i, j], P = softmax(Q K^T * scale);
+ * and, when avg != NULL, the "Avg" alternative avg_j = mean over heads and queries of P[n, i, j].
  */
 void pafu_oracle_sse_gmax(const uint16_t *Q, const uint16_t *K, int64_t L, int32_t N, int32_t D,
-                          double scale, double *g) {
+                          double scale, double *g, double *avg) {
     const int64_t dm = (int64_t)N * D;
-    for (int64_t j = 0; j < L; ++j) g[j] = 0.0;
+    for (int64_t j = 0; j < L; ++j) { g[j] = 0.0; if (avg) avg[j] = 0.0; }
     double *P = (double *)malloc(sizeof(double) * (size_t)L * (size_t)L);
     for (int32_t n = 0; n < N; ++n) {
 #pragma omp parallel for schedule(static)
@@ -352,6 +353,11 @@ void pafu_oracle_sse_gmax(const uint16_t *Q, const uint16_t *K, int64_t L, int32
             double mx = 0.0;
             for (int64_t i = 0; i < L; ++i) if (P[i * L + j] > mx) mx = P[i * L + j];
             g[j] += mx / N;
+            if (avg) {      /* the "Avg" alternative: mean over all queries */
+                double sm = 0.0;
+                for (int64_t i = 0; i < L; ++i) sm += P[i * L + j];
+                avg[j] += sm / L / N;
+            }
         }
     }
     free(P);

@@ -63,7 +63,7 @@ def _load():
                                         _c_f64p]
         lib.pafu_oracle_sse_gmax.restype = None
         lib.pafu_oracle_sse_gmax.argtypes = [_c_u16p, _c_u16p, ctypes.c_int64, ctypes.c_int32,
-                                             ctypes.c_int32, ctypes.c_double, _c_f64p]
+                                             ctypes.c_int32, ctypes.c_double, _c_f64p, _c_f64p]
         lib.pafu_oracle_sse_cols.restype = None
         lib.pafu_oracle_sse_cols.argtypes = [_c_u16p, _c_u16p, ctypes.c_int64, ctypes.c_int32,
                                              ctypes.c_int32, ctypes.c_int64, ctypes.c_double, _c_i64p,
@@ -197,5 +197,18 @@ def sse_global_max(Q: np.ndarray, K: np.ndarray, scale: Optional[float] = None) 
     if scale is None:
         scale = 1.0 / np.sqrt(D)
     g = np.empty(L, dtype=np.float64)
-    _load().pafu_oracle_sse_gmax(_p(Q, _c_u16p), _p(K, _c_u16p), L, N, D, float(scale), _p(g, _c_f64p))
+    _load().pafu_oracle_sse_gmax(_p(Q, _c_u16p), _p(K, _c_u16p), L, N, D, float(scale), _p(g, _c_f64p),
+                                 _p(None, _c_f64p))
     return g
+
+
+def sse_global_avg(Q: np.ndarray, K: np.ndarray, scale: Optional[float] = None) -> np.ndarray:
+    """Global average pooling of the attention weights (the "Avg" ablation, Sec. 4.3): [L]."""
+    Q = _u16(Q); K = _u16(K)
+    L, N, D = Q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    g = np.empty(L, dtype=np.float64); a = np.empty(L, dtype=np.float64)
+    _load().pafu_oracle_sse_gmax(_p(Q, _c_u16p), _p(K, _c_u16p), L, N, D, float(scale), _p(g, _c_f64p),
+                                 _p(a, _c_f64p))
+    return a

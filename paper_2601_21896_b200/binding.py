@@ -118,7 +118,7 @@ def lib() -> ctypes.CDLL:
         L.pafu_sse_workspace_bytes.restype = sz
         L.pafu_sse_workspace_bytes.argtypes = [i64, i32, i32, i64]
         L.pafu_sse.restype = i32
-        L.pafu_sse.argtypes = [vp, vp, vp, i64, i32, i32, i64, ctypes.c_float, vp, vp, vp, vp, sz, vp]
+        L.pafu_sse.argtypes = [vp, vp, vp, i64, i32, i32, i64, ctypes.c_float, vp, vp, vp, vp, vp, sz, vp]
         L.pafu_chunk_attn_noalloc.restype = i32
         L.pafu_chunk_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.POINTER(CShape),
                                               ctypes.c_float, vp, vp, vp]
@@ -299,12 +299,12 @@ def pafu_sse_workspace_bytes(L: int, n_heads: int, d_head: int, block_len: int) 
     return lib().pafu_sse_workspace_bytes(L, n_heads, d_head, block_len)
 
 
-def pafu_sse(Q, K, LSE, block_len: int, scale: float, s, comp, ws, gmax=None) -> None:
+def pafu_sse(Q, K, LSE, block_len: int, scale: float, s, comp, ws, gmax=None, gavg=None) -> None:
     """Teacher salience target (Eq. 4, Eq. 5) of Q, K [L, N, D]; LSE [N, L] or None; gmax [L]
-    (global max pooling) or None."""
+    (global max pooling) and gavg [L] (global average pooling) or None."""
     L, N, D = Q.shape
     _check(lib().pafu_sse(_ptr(Q), _ptr(K), _ptr(LSE), L, N, D, block_len, float(scale), _ptr(s), _ptr(comp),
-                          _ptr(gmax), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pafu_sse")
+                          _ptr(gmax), _ptr(gavg), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pafu_sse")
 
 
 def pafu_step_indexed(args: CStepArgs) -> None:

@@ -42,12 +42,12 @@ extern "C" size_t pafu_sse_workspace_bytes(int64_t L, int32_t n_heads, int32_t d
 
 extern "C" pafu_status pafu_sse(const uint16_t* Q, const uint16_t* K, const float* LSE, int64_t L,
                                 int32_t n_heads, int32_t d_head, int64_t block_len, float scale,
-                                float* s, float* comp, float* gmax, void* ws, size_t ws_bytes, void* stream) {
+                                float* s, float* comp, float* gmax, float* gavg, void* ws, size_t ws_bytes, void* stream) {
     if (!args_ok(L, n_heads, d_head, block_len)) return PAFU_ERR_INVALID_ARG;
     if (d_head != sse_tc::kD || L > 0x7fffffffLL) return PAFU_ERR_UNSUPPORTED_SHAPE;
     if (!(scale >= 0.f) || isinf(scale)) return PAFU_ERR_INVALID_ARG;
     if (Q == nullptr || K == nullptr || s == nullptr || ws == nullptr) return PAFU_ERR_INVALID_ARG;
-    if (!aligned16(Q) || !aligned16(K) || !aligned16(LSE) || !aligned16(s) || !aligned16(comp) || !aligned16(gmax)) return PAFU_ERR_MISALIGNED;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(LSE) || !aligned16(s) || !aligned16(comp) || !aligned16(gmax) || !aligned16(gavg)) return PAFU_ERR_MISALIGNED;
     if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
     const SsePlan pl = plan(L, n_heads, d_head, block_len);
     if (ws_bytes < pl.total) return PAFU_ERR_WORKSPACE_TOO_SMALL;
@@ -69,7 +69,7 @@ extern "C" pafu_status pafu_sse(const uint16_t* Q, const uint16_t* K, const floa
         if (e != PAFU_OK) return e;
         lse = lse_out;
     }
-    return sse_tc::launch(Q, K, lse, L, block_len, n_heads, scale, s, comp, gmax,
+    return sse_tc::launch(Q, K, lse, L, block_len, n_heads, scale, s, comp, gmax, gavg,
                           reinterpret_cast<uint16_t*>(base + pl.neglse), reinterpret_cast<float*>(base + pl.maxima),
                           reinterpret_cast<int*>(base) + kStatusWordTimeout, cs);
 }

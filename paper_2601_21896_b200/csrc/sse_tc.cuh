@@ -50,6 +50,7 @@ constexpr int kHalfBytes = kTileBytes / 2;     // one [128 rows x 64 cols] swizz
 constexpr int kAugBytes = kBT * 16 * 2;        // 4 KiB: 16 extra reduction columns of one tile
 constexpr int kStageBytes = kTileBytes + kAugBytes;   // Q tile, then its extra features
 constexpr int kSmemBytes = 2 * kTileBytes + kAugBytes + kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int kScratchRows = 4;               // low, diag, up maxima and the column sum, per head and key
 constexpr float kMasked = -1.0e30f;            // extra feature of a query column that does not exist
 
 struct Params {
@@ -62,7 +63,7 @@ struct Params {
     float sl2;                // scale * log2(e)
     float inv_scale;
     const uint16_t* q_aug;    // [n_heads][n_qt][2048] bf16: extra features per query tile, operand layout
-    float* M;                 // [n_heads][3][L]: per-head class maxima, log2 domain
+    float* M;                 // [n_heads][4][L]: per-head class maxima (log2 domain), then the column sums of P
     int* status;
 };
 
@@ -100,6 +101,8 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
+
+__device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 
 __device__ __forceinline__ uint16_t bf16_rne(float x) {
     const uint32_t u = __float_as_uint(x);
@@ -141,6 +144,9 @@ __global__ void sse_aug_kernel(const float* __restrict__ lse, Params p, uint16_t
     }
 }
 
+// SUM = true additionally accumulates sum_i P[i, j] per key (one exponential per element), for the
+// average-pooling output; the default instantiation does no exponentials at all.
+template <bool SUM>
 __global__ void __launch_bounds__(kThreads, 1)
 sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK,
               const __grid_constant__ Params p, int n_items) {
@@ -294,17 +300,23 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
             const bool w = mbar_wait(bar, ph) && !abort_flag;
             if (!__all_sync(0xffffffffu, w)) { if (lane == 0) fail(code); ok = false; }
         };
+        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;     // SUM: partial column sums of P for this key
         auto max64 = [&](const uint32_t (&r)[64], float& tm0, float& tm1) {
 #pragma unroll
             for (int q = 0; q < 16; ++q) {
                 tm0 = fmax3(tm0, __uint_as_float(r[4 * q + 0]), __uint_as_float(r[4 * q + 1]));
                 tm1 = fmax3(tm1, __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+                if (SUM) {
+                    sum0 += ex2(__uint_as_float(r[4 * q + 0]) * p.sl2); sum1 += ex2(__uint_as_float(r[4 * q + 1]) * p.sl2);
+                    sum2 += ex2(__uint_as_float(r[4 * q + 2]) * p.sl2); sum3 += ex2(__uint_as_float(r[4 * q + 3]) * p.sl2);
+                }
             }
         };
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const Item it = decode_item(p, item);
             if (slot >= it.n_slots) continue;
             float m_low = -INFINITY, m_diag = -INFINITY, m_up = -INFINITY;
+            sum0 = sum1 = sum2 = sum3 = 0.f;
             uint32_t ra[64], rb[64];
             wait_warp(s_full(slot, tc & 1), (tc >> 1) & 1u, 522);
             if (!ok) break;
@@ -346,8 +358,9 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
             const int64_t key = it.key0 + slot * kBT + row_in_tile;
             if (key < it.block_end) {
                 // log2 domain; a class without queries stays -inf, a masked column gives about -1e29
-                float* dst = p.M + (int64_t)it.head * 3 * p.L + key;
+                float* dst = p.M + (int64_t)it.head * kScratchRows * p.L + key;
                 dst[0] = m_low * p.sl2; dst[p.L] = m_diag * p.sl2; dst[2 * p.L] = m_up * p.sl2;
+                if (SUM) dst[3 * p.L] = (sum0 + sum1) + (sum2 + sum3);
             }
         }
         if (!ok) tmem_wait_ld();      // no load may be in flight when tensor memory is released
@@ -358,14 +371,15 @@ sse_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
 }
 
 // exp2 of the per-head maxima, mean over heads (head order), Eq. 5.
-__global__ void sse_finish_kernel(Params p, float* __restrict__ s, float* __restrict__ comp, float* __restrict__ gmax) {
+__global__ void sse_finish_kernel(Params p, float* __restrict__ s, float* __restrict__ comp, float* __restrict__ gmax,
+                                  float* __restrict__ gavg) {
     grid_dep_wait();
     for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < p.L; j += (int64_t)gridDim.x * blockDim.x) {
         float c[3];
 #pragma unroll
         for (int k = 0; k < 3; ++k) {
             float acc = 0.f;
-            for (int n = 0; n < p.n_heads; ++n) acc += exp2f(p.M[((int64_t)n * 3 + k) * p.L + j]);
+            for (int n = 0; n < p.n_heads; ++n) acc += exp2f(p.M[((int64_t)n * kScratchRows + k) * p.L + j]);
             c[k] = acc / (float)p.n_heads;
         }
         float v;
@@ -377,10 +391,15 @@ __global__ void sse_finish_kernel(Params p, float* __restrict__ s, float* __rest
         if (gmax != nullptr) {          // max over all queries per head, then the mean over heads
             float acc = 0.f;
             for (int n = 0; n < p.n_heads; ++n) {
-                const float* m = p.M + (int64_t)n * 3 * p.L + j;
+                const float* m = p.M + (int64_t)n * kScratchRows * p.L + j;
                 acc += exp2f(fmaxf(fmaxf(m[0], m[p.L]), m[2 * p.L]));
             }
             gmax[j] = acc / (float)p.n_heads;
+        }
+        if (gavg != nullptr) {          // mean over all queries per head, then the mean over heads
+            float acc = 0.f;
+            for (int n = 0; n < p.n_heads; ++n) acc += p.M[((int64_t)n * kScratchRows + 3) * p.L + j];
+            gavg[j] = acc / ((float)p.n_heads * (float)p.L);
         }
     }
 }
@@ -403,10 +422,10 @@ inline Params make_params(int64_t L, int64_t LB, int n_heads, float scale) {
 }
 
 inline size_t aug_bytes(const Params& p) { return (size_t)p.n_heads * p.n_qt * kAugBytes; }
-inline size_t maxima_bytes(const Params& p) { return (size_t)p.n_heads * 3 * p.L * 4; }
+inline size_t maxima_bytes(const Params& p) { return (size_t)p.n_heads * kScratchRows * p.L * 4; }
 
 inline pafu_status launch(const uint16_t* Q, const uint16_t* K, const float* lse, int64_t L, int64_t LB,
-                          int n_heads, float scale, float* s, float* comp, float* gmax, uint16_t* q_aug, float* M,
+                          int n_heads, float scale, float* s, float* comp, float* gmax, float* gavg, uint16_t* q_aug, float* M,
                           int* status, cudaStream_t stream) {
     Params p = make_params(L, LB, n_heads, scale);
     p.q_aug = q_aug; p.M = M; p.status = status;
@@ -415,7 +434,8 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* K, const float* lse
         !TmapEncoder::token_tensor(&mK, K, (uint64_t)L, n_heads, kD, kBT)) return PAFU_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(sse_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(sse_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(sse_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return PAFU_ERR_CUDA;
         attr_set = true;
     }
@@ -426,10 +446,11 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* K, const float* lse
         return PAFU_ERR_CUDA;
     const int n_items = n_heads * p.items_per_head;
     const int grid = n_items < sms ? n_items : sms;
-    if (launch_dependent(sse_tc_kernel, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mK, p, n_items) != cudaSuccess)
+    if ((gavg != nullptr ? launch_dependent(sse_tc_kernel<true>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mK, p, n_items)
+                         : launch_dependent(sse_tc_kernel<false>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mK, p, n_items)) != cudaSuccess)
         return PAFU_ERR_CUDA;
     const int g2 = (int)((L + 255) / 256 < 4 * sms ? (L + 255) / 256 : 4 * sms);
-    if (launch_dependent(sse_finish_kernel, dim3(g2), dim3(256), 0, stream, 1, p, s, comp, gmax) != cudaSuccess)
+    if (launch_dependent(sse_finish_kernel, dim3(g2), dim3(256), 0, stream, 1, p, s, comp, gmax, gavg) != cudaSuccess)
         return PAFU_ERR_CUDA;
     return PAFU_OK;
 }

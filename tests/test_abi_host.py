@@ -125,7 +125,7 @@ def test_newer_entry_points_reject_bad_arguments_on_host(L):
     assert cl((ctypes.c_void_p * 2)(fake, None), 2, out) == 1       # a missing layer
     assert cl(arr, 0, out) == 0                                     # no layers: no-op
     # teacher salience target
-    sse = lambda Lt, N, D, LB, scale, s, ws, nb: L.pafu_sse(fake, fake, None, Lt, N, D, LB, scale, s, None, None, ws, nb, None)
+    sse = lambda Lt, N, D, LB, scale, s, ws, nb: L.pafu_sse(fake, fake, None, Lt, N, D, LB, scale, s, None, None, None, ws, nb, None)
     need = L.pafu_sse_workspace_bytes(1000, 2, 128, 256)
     assert need > 0 and need % 256 == 0
     assert L.pafu_sse_workspace_bytes(1000, 2, 64, 256) == 0 and L.pafu_sse_workspace_bytes(0, 2, 128, 256) == 0

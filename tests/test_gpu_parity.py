@@ -364,10 +364,12 @@ def test_sse_matches_oracle(L, N, LB):
     ws = torch.zeros(pafu.pafu_sse_workspace_bytes(L, N, D, LB), dtype=torch.uint8, device="cuda")
     s = torch.full((L,), float("nan"), device="cuda"); comp = torch.full((3, L), float("nan"), device="cuda")
     gmax = torch.full((L,), float("nan"), device="cuda")
-    pafu.pafu_sse(dQ, dK, None, LB, 0.0, s, comp, ws, gmax=gmax)
+    gavg = torch.full((L,), float("nan"), device="cuda")
+    pafu.pafu_sse(dQ, dK, None, LB, 0.0, s, comp, ws, gmax=gmax, gavg=gavg)
     assert pafu.pafu_workspace_status(ws) == 0
     tol = dict(rtol=1e-3, atol=1e-7)
     assert np.allclose(gmax.cpu().numpy(), oracle.sse_global_max(Q, K), **tol)    # the "Max" ablation
+    assert np.allclose(gavg.cpu().numpy(), oracle.sse_global_avg(Q, K), **tol)    # the "Avg" ablation
     assert np.allclose(comp.cpu().numpy(), want_c, **tol), np.abs(comp.cpu().numpy() - want_c).max()
     assert np.allclose(s.cpu().numpy(), want_s, **tol)
     # with the row statistics handed in (as the attention call leaves them) the result is the same

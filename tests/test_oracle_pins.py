@@ -402,6 +402,9 @@ def test_sse_global_max_against_dense_torch():
     tq = torch.from_numpy(f32(Q)).double(); tk = torch.from_numpy(f32(K)).double()
     P = torch.softmax(torch.einsum("qnd,knd->nqk", tq, tk) / math.sqrt(D), dim=-1)
     assert np.allclose(g, P.max(dim=1).values.mean(dim=0).numpy(), atol=1e-14)
+    a = oracle.sse_global_avg(Q, K)
+    assert np.allclose(a, P.mean(dim=1).mean(dim=0).numpy(), atol=1e-14)
+    assert abs(a.sum() - 1.0) < 1e-12          # rows of P sum to one, so the column means sum to one
     # it dominates each of the three block-wise components and equals their maximum for one head
     _, comp = oracle.sse(Q[:, :1], K[:, :1], 5)
     assert np.allclose(oracle.sse_global_max(Q[:, :1], K[:, :1]), comp.max(axis=0), atol=1e-14)
