@@ -541,6 +541,13 @@ def run_ours(args):
         "shared_index_compaction": shared,
         "layers_per_step": n_layers,
         "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step / n_layers,
+        # the paper's own schedule (Sec. 3.3, Algorithm 2): score the new chunk and prune every layer's
+        # cache once per chunk with the final layer's indices; every denoising step then only attends
+        "paper_schedule": None if not (qkv and shared and args.shared_layers == N_LAYERS_PER_DENOISE_STEP) else {
+            "prune_once_per_chunk_ms": qkv["ms"] + shared["ms"],
+            "attention_per_denoise_step_30_layers_ms": N_LAYERS_PER_DENOISE_STEP * float(k_ms[3]),
+            "note": "S-MLP on the chunk's [q,k,v] + one select + 30-layer shared-index compaction; "
+                    "30 x (attention + merge) per denoising step"},
         "peaks": peaks,
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
