@@ -7,7 +7,7 @@
 // 128-row "slots" that share every K/V tile (each tile is fetched once per 256 rows).  The
 // grid is persistent: one CTA per SM.  All items' key tiles are laid end to end and cut into
 // equal contiguous shares, one per CTA (a tile with both slots live costs 8 units, with one
-// slot 7: a lone slot has no partner to hide its softmax behind), so every SM gets the same
+// slot 6: a lone slot has no partner to hide its softmax behind), so every SM gets the same
 // amount of work whatever the item count.  A CTA whose share covers only
 // part of an item's keys writes an unnormalised partial (O, running max, row sum) to the
 // workspace; a second small kernel merges the partials of each split item in key order, which
@@ -92,7 +92,7 @@ struct Seg {
                          // earlier CTA; 1: begins an item that a later CTA continues
 };
 
-constexpr int kCost2 = 8, kCost1 = 7;   // cost of one key tile with two / one live slots (measured ratio)
+constexpr int kCost2 = 8, kCost1 = 6;   // cost of one key tile with two / one live slots (best of 5..7 on every measured workload)
 
 struct StreamCost {
     int64_t nqp, nt, head_cost;
