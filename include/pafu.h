@@ -204,14 +204,15 @@ pafu_status pafu_chunk_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_
  * ("index-based cache management": Sec. 3.4, Eq. 7 restricts attention to the index set I_s of the
  * full cache instead of to a copied cache).  Computes exactly what pafu_compact followed by
  * pafu_chunk_attn computes - the outputs are bit-identical - but K and V are the UNCOMPACTED
- * cache and the loader fetches rows idx[.] of it, so no compacted copy is written or read.
+ * cache and the loader fetches rows idx[.] of it, so no compacted copy is written or read (the
+ * attention itself runs about a tenth slower than on a compacted cache).
  *   K, V      device bf16 [cu_T[n_streams], n_heads, d_head], the cache before pruning
  *   idx       device int32 [cu_B[n_streams]] as written by pafu_select: per stream, stream-local
  *             token indices in [0, T_s), at offset cu_B[s]
  *   cu_B      HOST prefix array of retained tokens (pafu_kept_counts); B_s <= T_s
  *   shape     needs both cu_T and cu_Lq
  * Everything else as pafu_chunk_attn.  Supported: d_head = 128; every stream with queries needs
- * at least one key; total cache rows < 2^31. */
+ * at least one key; K and V smaller than 64 GiB each. */
 pafu_status pafu_chunk_attn_indexed(const uint16_t* Q, const uint16_t* K, const uint16_t* V, const int32_t* idx,
                                     const int64_t* cu_B, const uint16_t* Kq, const uint16_t* Vq,
                                     const pafu_shape* shape, float scale, uint16_t* O, float* LSE,

@@ -281,7 +281,9 @@ pafu_status pafu_chunk_attn_indexed(const uint16_t* Q, const uint16_t* K, const 
     for (int s = 0; s < st.n_streams; ++s) {
         if (st.cu_B[s + 1] - st.cu_B[s] > st.cu_T[s + 1] - st.cu_T[s]) return PAFU_ERR_INVALID_ARG;
     }
-    if (st.cu_T[st.n_streams] > 0x7fffffffLL) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    // the loader addresses cache rows with 32-bit offsets in 16-byte units: K and V below 64 GiB each
+    if (st.cu_T[st.n_streams] > 0x7fffffffLL ||
+        (uint64_t)st.cu_T[st.n_streams] * (uint64_t)shape->n_heads * 16u >= (1ull << 32)) return PAFU_ERR_UNSUPPORTED_SHAPE;
     if (st.cu_Lq[st.n_streams] == 0) return PAFU_OK;
     if (Q == nullptr || O == nullptr) return PAFU_ERR_INVALID_ARG;
     if ((Kq == nullptr) != (Vq == nullptr)) return PAFU_ERR_INVALID_ARG;

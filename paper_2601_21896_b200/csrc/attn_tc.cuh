@@ -78,6 +78,8 @@ struct Params {
     int* status;        // workspace status word (device)
     float* pieces;      // [gridDim][2][kPieceFloats]
     const int32_t* idx; // gather variant: retained token indices, stream-local, [cu_B[n_streams]]
+    const uint16_t* Kraw;   // gather variant: the uncompacted cache [cu_T[n_streams], n_heads, 128]
+    const uint16_t* Vraw;
     int64_t total_Lq;
     int64_t total_cost;
 };
@@ -199,8 +201,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 // GATHER = false: the retained keys/values are the rows of a compacted cache (mKc, mVc are tiled
 // maps of it).  GATHER = true: they are rows idx[.] of the uncompacted cache, fetched by the
-// loader four rows at a time (mKc, mVc are two-dimensional [tokens, n_heads * d_head] maps with a
-// one-row box); everything downstream of the shared-memory ring is identical.
+// loader warp with 16-byte asynchronous copies (mKc, mVc unused); everything downstream of the
+// shared-memory ring is identical.
 template <bool GATHER>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mKc,
@@ -235,7 +237,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
             mbar_init(pv_done(s), 1); mbar_init(o_done(s), 1);
         }
         for (int st = 0; st < kStages; ++st) {
-            mbar_init(kv_full(st), 1);
+            mbar_init(kv_full(st), GATHER ? 32 : 1);    // gather: every lane of the loader warp arrives
             mbar_init(kv_empty(st), 2);                 // both issuers release a stage
         }
         abort_flag = 0;
@@ -256,82 +258,92 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
     if (warp >= 8) {
     // register budget: this warpgroup gives registers up, the softmax warpgroups take them
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLow));
-    if (warp == 11) {
+    if (warp == 11 && !GATHER) {
         // idle
-    } else if (warp == 9) {
+    } else if (warp == 9 || warp == 11) {
         // ------------------------------------------------------------------ TMA loader
         if constexpr (GATHER) {
-            // The whole warp walks the runs together.  Lane 0 issues the tiled loads (Q, the
-            // chunk's own K/V); a retained 64-key tile is 2 column halves x 16 groups of four
-            // rows, one gather per lane for K and one for V, each writing 4 x 128 bytes at the
-            // place the tiled load would have put those rows (the swizzle is a function of the
-            // shared-memory address, so the tile's layout is unchanged).
+            // Two loader warps walk the runs together: warp 9 fills the K stages of the ring (and
+            // loads Q), warp 11 the V stages.  Lane 0 issues the tiled loads (Q, the chunk's own
+            // K/V).  A retained 64-key tile is fetched with 16-byte asynchronous copies: a lane owns
+            // one 16-byte piece of a 128-byte row segment (8 pieces x 2 column halves x 2 rows per
+            // warp instruction, 32 instructions per tile) and writes it where the tiled load would
+            // have put it (128-byte swizzle: piece c of row r goes to piece c ^ (r mod 8)), so the
+            // operand layout is unchanged.  The tile's 64 row offsets (in 16-byte units) sit in
+            // two registers per lane and are handed round by shuffles.
             const int lane = tid & 31;
-            const int grp = lane & 15, half = lane >> 4;
+            const int kv = warp == 9 ? 0 : 1;
+            const int r2 = lane >> 4, half = (lane >> 3) & 1, piece = lane & 7;
             if (lane == 0) {
-                prefetch_tmap(&mQ); prefetch_tmap(&mKc); prefetch_tmap(&mVc);
-                if (p.has_chunk) { prefetch_tmap(&mKq); prefetch_tmap(&mVq); }
+                if (kv == 0) prefetch_tmap(&mQ);
+                if (p.has_chunk) prefetch_tmap(kv ? &mVq : &mKq);
             }
             SegIter iter(p, blockIdx.x, gridDim.x);
             Seg g;
-            uint32_t ring = 0, qcnt0 = 0, qcnt1 = 0;
+            uint32_t ring = (uint32_t)kv, qcnt0 = 0, qcnt1 = 0;     // this warp's stages: every other ring entry
             bool ok = true;
             auto wait_all = [&](uint32_t bar, uint32_t ph, int code) {
                 const bool w = !abort_flag && mbar_wait(bar, ph);
                 if (!__all_sync(0xffffffffu, w)) { if (lane == 0) fail(code); ok = false; }
             };
+            const uint32_t row16 = (uint32_t)p.n_heads * (kD * 2 / 16);          // 16-byte units per token row
+            const uint32_t lane_dst = (uint32_t)(half * kHalfBytes + r2 * 128);
+            const uint32_t sw = (uint32_t)(piece ^ r2);                          // piece ^ (row & 7) = sw ^ ((2 it) & 7)
             while (ok && iter.next(p, g)) {
-                const int qrow = (int)(p.st.cu_Lq[g.stream] + g.q0);
-                for (int s = 0; s < g.n_slots && ok; ++s) {
-                    const uint32_t qc = s ? qcnt1 : qcnt0;
-                    wait_all(q_empty(s), (qc & 1u) ^ 1u, 100);
-                    if (!ok) break;
-                    if (s) ++qcnt1; else ++qcnt0;
-                    if (lane == 0) {
-                        mbar_arrive_expect_tx(q_full(s), kQBytes);
-                        tma_load_3d(sQ + s * kQBytes, &mQ, q_full(s), 0, g.head, qrow + s * kBM);
-                        tma_load_3d(sQ + s * kQBytes + kQHalf, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
+                if (kv == 0) {
+                    const int qrow = (int)(p.st.cu_Lq[g.stream] + g.q0);
+                    for (int s = 0; s < g.n_slots && ok; ++s) {
+                        const uint32_t qc = s ? qcnt1 : qcnt0;
+                        wait_all(q_empty(s), (qc & 1u) ^ 1u, 100);
+                        if (!ok) break;
+                        if (s) ++qcnt1; else ++qcnt0;
+                        if (lane == 0) {
+                            mbar_arrive_expect_tx(q_full(s), kQBytes);
+                            tma_load_3d(sQ + s * kQBytes, &mQ, q_full(s), 0, g.head, qrow + s * kBM);
+                            tma_load_3d(sQ + s * kQBytes + kQHalf, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
+                        }
                     }
                 }
                 const int32_t* sidx = p.idx + p.st.cu_B[g.stream];
                 const int row_base = (int)p.st.cu_T[g.stream];
-                for (int j = g.t0; j < g.t1 && ok; ++j) {
+                const uint8_t* base = reinterpret_cast<const uint8_t*>(kv ? p.Vraw : p.Kraw) +
+                                      (size_t)g.head * (kD * 2) + half * 128 + piece * 16;
+                for (int j = g.t0; j < g.t1 && ok; ++j, ring += 2) {
                     const bool seg2 = j >= g.nt1;
-                    int r[4] = {0, 0, 0, 0};
+                    const int st = ring % kStages;
+                    uint32_t o0 = 0, o1 = 0;
                     if (!seg2) {
                         // rows past the segment's end repeat its last row: their logits are masked,
                         // and their values must be finite
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            int64_t pos = (int64_t)j * kBN + grp * 4 + e;
-                            if (pos >= g.nB) pos = g.nB - 1;
-                            r[e] = row_base + __ldg(sidx + pos);
-                        }
+                        int64_t pos = (int64_t)j * kBN + lane;
+                        o0 = (uint32_t)(row_base + __ldg(sidx + (pos < g.nB ? pos : g.nB - 1))) * row16;
+                        pos += 32;
+                        o1 = (uint32_t)(row_base + __ldg(sidx + (pos < g.nB ? pos : g.nB - 1))) * row16;
                     }
-                    const int row2 = (int)(p.st.cu_Lq[g.stream] + (int64_t)(j - g.nt1) * kBN);
-                    for (int kv = 0; kv < 2 && ok; ++kv, ++ring) {
-                        const int st = ring % kStages;
-                        wait_all(kv_empty(st), ((ring / kStages) & 1u) ^ 1u, 101);
-                        if (!ok) break;
-                        if (lane == 0) mbar_arrive_expect_tx(kv_full(st), kTileBytes);
-                        __syncwarp();
-                        if (seg2) {
-                            if (lane == 0) {
-                                const CUtensorMap* m = kv ? &mVq : &mKq;
-                                tma_load_3d(sKV + st * kTileBytes, m, kv_full(st), 0, g.head, row2);
-                                tma_load_3d(sKV + st * kTileBytes + kHalfBytes, m, kv_full(st), 64, g.head, row2);
-                            }
+                    wait_all(kv_empty(st), ((ring / kStages) & 1u) ^ 1u, 101);
+                    if (!ok) break;
+                    if (seg2) {
+                        if (lane == 0) {
+                            const CUtensorMap* m = kv ? &mVq : &mKq;
+                            const int row2 = (int)(p.st.cu_Lq[g.stream] + (int64_t)(j - g.nt1) * kBN);
+                            mbar_arrive_expect_tx(kv_full(st), kTileBytes);
+                            tma_load_3d(sKV + st * kTileBytes, m, kv_full(st), 0, g.head, row2);
+                            tma_load_3d(sKV + st * kTileBytes + kHalfBytes, m, kv_full(st), 64, g.head, row2);
                         } else {
-                            tma_gather4_2d(sKV + st * kTileBytes + half * kHalfBytes + grp * 512, kv ? &mVc : &mKc,
-                                           kv_full(st), g.head * kD + half * 64, r[0], r[1], r[2], r[3]);
+                            mbar_arrive(kv_full(st));
                         }
+                    } else {
+                        const uint32_t dst0 = sKV + st * kTileBytes + lane_dst;
+#pragma unroll
+                        for (int it = 0; it < kBN / 2; ++it) {
+                            const uint32_t off16 = __shfl_sync(0xffffffffu, it < 16 ? o0 : o1, (2 * it + r2) & 31);
+                            cp_async_16(dst0 + it * 256 + ((sw ^ (uint32_t)((2 * it) & 7)) << 4), base + (size_t)off16 * 16);
+                        }
+                        cp_async_mbar_arrive_noinc(kv_full(st));
                     }
                 }
             }
-            if (!ok) {
-                for (uint32_t r = ring > (uint32_t)kStages ? ring - kStages : 0; r < ring; ++r)
-                    mbar_wait(kv_full(r % kStages), (r / kStages) & 1u);
-            }
+            cp_async_wait_all();
         } else if (elect_one()) {
             prefetch_tmap(&mQ); prefetch_tmap(&mKc); prefetch_tmap(&mVc);
             if (p.has_chunk) { prefetch_tmap(&mKq); prefetch_tmap(&mVq); }
@@ -437,6 +449,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 for (int i = 0; i < 2 && i < n && ok; ++i) {        // S(0), S(1)
                     wait(kv_full(ck.st), ck.ph, 202);
                     if (!ok) break;
+                    if constexpr (GATHER) fence_proxy_async_smem();   // the tile came through the generic proxy
                     tc_fence_after_sync();
                     issue_qk((tc + i) & 1, ck.st);
                     umma_commit(s_full(slot, (tc + i) & 1));
@@ -450,12 +463,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                     wait(kv_full(cv.st), cv.ph, 203);
                     if (!ok) break;
                     if (!mbar_wait_spin(p_full(slot, buf), ((tc + i) >> 1) & 1u)) { fail(205); ok = false; break; }
+                    if constexpr (GATHER) fence_proxy_async_smem();
                     tc_fence_after_sync();
                     issue_pv(buf, cv.st, i == 0);
                     umma_commit(kv_empty(cv.st));
                     if (i + 2 < n) {                                // S(i+2) reuses the buffer P(i) was read from
                         wait(kv_full(ck.st), ck.ph, 204);
                         if (!ok) break;
+                        if constexpr (GATHER) fence_proxy_async_smem();
                         issue_qk(buf, ck.st);
                         umma_commit(s_full(slot, buf));
                         umma_commit(kv_empty(ck.st));
@@ -809,8 +824,8 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
     if (!TmapEncoder::token_tensor(&mQ, Q, (uint64_t)nQ, n_heads, kD, kBM)) return PAFU_ERR_CUDA;
     const bool gather = idx != nullptr;      // Kc, Vc are then the uncompacted cache of n_cache_rows tokens
     if (nB > 0 && gather) {
-        if (!TmapEncoder::matrix(&mKc, Kc, (uint64_t)n_cache_rows, (uint64_t)n_heads * kD, (uint64_t)n_heads * kD, 1) ||
-            !TmapEncoder::matrix(&mVc, Vc, (uint64_t)n_cache_rows, (uint64_t)n_heads * kD, (uint64_t)n_heads * kD, 1)) return PAFU_ERR_CUDA;
+        mKc = mQ; mVc = mQ;                 // the gather loader reads the cache through plain pointers
+        (void)n_cache_rows;
     } else if (nB > 0) {
         if (!TmapEncoder::token_tensor(&mKc, Kc, (uint64_t)nB, n_heads, kD, kBN) ||
             !TmapEncoder::token_tensor(&mVc, Vc, (uint64_t)nB, n_heads, kD, kBN)) return PAFU_ERR_CUDA;
@@ -821,7 +836,7 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
     } else { mKq = mQ; mVq = mQ; }
     Params p;
     p.st = st; p.n_heads = n_heads; p.has_chunk = has_chunk; p.scale = scale;
-    p.O = O; p.LSE = LSE; p.status = status; p.pieces = pieces; p.idx = idx; p.total_Lq = nQ; p.total_cost = cost;
+    p.O = O; p.LSE = LSE; p.status = status; p.pieces = pieces; p.idx = idx; p.Kraw = gather ? Kc : nullptr; p.Vraw = gather ? Vc : nullptr; p.total_Lq = nQ; p.total_cost = cost;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
