@@ -266,14 +266,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
             // Two loader warps walk the runs together: warp 9 fills the K stages of the ring (and
             // loads Q), warp 11 the V stages.  Lane 0 issues the tiled loads (Q, the chunk's own
             // K/V).  A retained 64-key tile is fetched with 16-byte asynchronous copies: a lane owns
-            // one 16-byte piece of a 128-byte row segment (8 pieces x 2 column halves x 2 rows per
-            // warp instruction, 32 instructions per tile) and writes it where the tiled load would
-            // have put it (128-byte swizzle: piece c of row r goes to piece c ^ (r mod 8)), so the
-            // operand layout is unchanged.  The tile's 64 row offsets (in 16-byte units) sit in
-            // two registers per lane and are handed round by shuffles.
+            // 16-byte pieces c and c + 4 of a row in both 64-column halves (4 lanes per row, 8 rows
+            // per warp instruction, 4 x 8 instructions per tile) and writes them where the tiled load
+            // would have put them (128-byte swizzle: piece c of row r goes to piece c ^ (r mod 8)),
+            // so the operand layout is unchanged.  The tile's 64 row offsets (in 16-byte units) sit
+            // in two registers per lane, are handed round by shuffles and are fetched one tile
+            // ahead of their use.
             const int lane = tid & 31;
             const int kv = warp == 9 ? 0 : 1;
-            const int r2 = lane >> 4, half = (lane >> 3) & 1, piece = lane & 7;
+            const int r8 = lane >> 2, piece = lane & 3;           // row within a group of eight; pieces `piece` and `piece + 4`
             if (lane == 0) {
                 if (kv == 0) prefetch_tmap(&mQ);
                 if (p.has_chunk) prefetch_tmap(kv ? &mVq : &mKq);
@@ -287,8 +288,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 if (!__all_sync(0xffffffffu, w)) { if (lane == 0) fail(code); ok = false; }
             };
             const uint32_t row16 = (uint32_t)p.n_heads * (kD * 2 / 16);          // 16-byte units per token row
-            const uint32_t lane_dst = (uint32_t)(half * kHalfBytes + r2 * 128);
-            const uint32_t sw = (uint32_t)(piece ^ r2);                          // piece ^ (row & 7) = sw ^ ((2 it) & 7)
+            // row = 8 it + r8, so row & 7 = r8: a lane's two swizzled positions never change
+            const uint32_t dst_a = (uint32_t)(r8 * 128 + ((piece ^ r8) << 4));
+            const uint32_t dst_b = (uint32_t)(r8 * 128 + (((piece + 4) ^ r8) << 4));
             while (ok && iter.next(p, g)) {
                 if (kv == 0) {
                     const int qrow = (int)(p.st.cu_Lq[g.stream] + g.q0);
@@ -307,19 +309,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 const int32_t* sidx = p.idx + p.st.cu_B[g.stream];
                 const int row_base = (int)p.st.cu_T[g.stream];
                 const uint8_t* base = reinterpret_cast<const uint8_t*>(kv ? p.Vraw : p.Kraw) +
-                                      (size_t)g.head * (kD * 2) + half * 128 + piece * 16;
-                for (int j = g.t0; j < g.t1 && ok; ++j, ring += 2) {
-                    const bool seg2 = j >= g.nt1;
-                    const int st = ring % kStages;
-                    uint32_t o0 = 0, o1 = 0;
-                    if (!seg2) {
-                        // rows past the segment's end repeat its last row: their logits are masked,
-                        // and their values must be finite
+                                      (size_t)g.head * (kD * 2) + piece * 16;
+                // row offsets of a retained tile (rows past the segment's end repeat its last row:
+                // their logits are masked, and their values must be finite)
+                auto tile_offsets = [&](int j, uint32_t& o0, uint32_t& o1) {
+                    o0 = o1 = 0;
+                    if (j < g.t1 && j < g.nt1) {
                         int64_t pos = (int64_t)j * kBN + lane;
                         o0 = (uint32_t)(row_base + __ldg(sidx + (pos < g.nB ? pos : g.nB - 1))) * row16;
                         pos += 32;
                         o1 = (uint32_t)(row_base + __ldg(sidx + (pos < g.nB ? pos : g.nB - 1))) * row16;
                     }
+                };
+                uint32_t o0, o1, n0, n1;
+                tile_offsets(g.t0, o0, o1);
+                for (int j = g.t0; j < g.t1 && ok; ++j, ring += 2) {
+                    const bool seg2 = j >= g.nt1;
+                    const int st = ring % kStages;
+                    tile_offsets(j + 1, n0, n1);                     // the next tile's indices, one tile ahead
                     wait_all(kv_empty(st), ((ring / kStages) & 1u) ^ 1u, 101);
                     if (!ok) break;
                     if (seg2) {
@@ -333,14 +340,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                             mbar_arrive(kv_full(st));
                         }
                     } else {
-                        const uint32_t dst0 = sKV + st * kTileBytes + lane_dst;
+                        const uint32_t dst0 = sKV + st * kTileBytes;
 #pragma unroll
-                        for (int it = 0; it < kBN / 2; ++it) {
-                            const uint32_t off16 = __shfl_sync(0xffffffffu, it < 16 ? o0 : o1, (2 * it + r2) & 31);
-                            cp_async_16(dst0 + it * 256 + ((sw ^ (uint32_t)((2 * it) & 7)) << 4), base + (size_t)off16 * 16);
+                        for (int it = 0; it < kBN / 8; ++it) {
+                            const uint32_t off16 = __shfl_sync(0xffffffffu, it < 4 ? o0 : o1, (8 * it + r8) & 31);
+                            const uint8_t* src = base + (size_t)off16 * 16;
+                            const uint32_t d = dst0 + it * 1024;
+                            cp_async_16(d + dst_a, src);                                // columns 0..63
+                            cp_async_16(d + dst_b, src + 64);
+                            cp_async_16(d + dst_a + kHalfBytes, src + 128);             // columns 64..127
+                            cp_async_16(d + dst_b + kHalfBytes, src + 192);
                         }
                         cp_async_mbar_arrive_noinc(kv_full(st));
                     }
+                    o0 = n0; o1 = n1;
                 }
             }
             cp_async_wait_all();
