@@ -331,8 +331,9 @@ def test_indexed_attention_matches_oracle_and_compacted_path():
         assert torch.equal(O.view(torch.int16), O2.view(torch.int16)) and torch.equal(LSE, LSE2)
 
 
-@pytest.mark.parametrize("w", [wl.small_ragged(2, 128), wl.wan13b_layer(), wl.batch4_14b()],
-                         ids=lambda w: w.name)
+@pytest.mark.parametrize("w", [wl.small_ragged(2, 128), wl.wan13b_layer(), wl.wan13b_layer(0.25), wl.paper_native(),
+                               wl.long_horizon(), wl.batch4_14b()],
+                         ids=lambda w: "%s-B%d" % (w.name, w.budget[0]))
 def test_step_indexed_equals_step(w):
     d = wl.make_layer(w)
     A = Layer(w, d); B = Layer(w, d)
