@@ -118,6 +118,23 @@ size_t pafu_workspace_bytes(const pafu_shape* shape, const pafu_policy* policy,
  * the header was last zeroed (the outputs of that launch are then undefined). */
 pafu_status pafu_workspace_status(const void* ws, void* stream);
 
+/* Diagnostic counters of the workspace's status header, accumulated by pafu_chunk_attn (d_head
+ * 128) since the header was last zeroed.  SYNCHRONISES `stream`.  The attention kernel keeps a
+ * running row maximum per query (the max-subtracted softmax of Sec. 3.2 evaluated tile by tile)
+ * and only re-bases it when it must; the counters say how often each path ran, counted per
+ * (32-row group, 64-key tile):
+ *   counts[0]  tiles that took the exact pass because they open a run or end a key segment raggedly
+ *   counts[1]  tiles that took the exact pass because a row sum showed a logit far above the
+ *              running maximum
+ *   counts[2]  tiles at which the output accumulator and the row sums were rescaled
+ * counts is a HOST array of 3 entries.  Tests use it to show that an input reaches those paths.
+ *
+ * The header also holds a test hook: while its 32-bit word 32 is non-zero the attention kernel's
+ * loader issues no copies, every consumer's bounded wait runs out and the launch ends with
+ * PAFU_ERR_TIMEOUT in the header (outputs undefined).  It exists so that the time-out path can
+ * be exercised without faulting the device; zero the header to return to normal operation. */
+pafu_status pafu_workspace_counters(const void* ws, int64_t* counts, void* stream);
+
 /* Step 1 - salience scores (Sec. 3.3, 3.4; Appendix A "S-MLP").
  * For every token row x of X: h = act(W1 x + b1); y = W2 h + b2; s = mean_o y_o;
  * s <- sigmoid(s) if head->final == PAFU_FINAL_SIGMOID.  bf16 operands, fp32 accumulation,

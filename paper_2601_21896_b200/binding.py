@@ -27,7 +27,7 @@ STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET
                 8: "PAFU_ERR_TOO_LARGE"}
 
 EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
-           "pafu_workspace_status", "pafu_score", "pafu_score_qkv", "pafu_select", "pafu_compact",
+           "pafu_workspace_status", "pafu_workspace_counters", "pafu_score", "pafu_score_qkv", "pafu_select", "pafu_compact",
            "pafu_chunk_attn", "pafu_chunk_attn_indexed", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_indexed", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host",
            "pafu_sse_workspace_bytes", "pafu_sse", "pafu_compact_layers"]
 
@@ -95,6 +95,8 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(CHead)]
         L.pafu_workspace_status.restype = i32
         L.pafu_workspace_status.argtypes = [vp, vp]
+        L.pafu_workspace_counters.restype = i32
+        L.pafu_workspace_counters.argtypes = [vp, vp, vp]
         L.pafu_score.restype = i32
         L.pafu_score.argtypes = [ctypes.POINTER(CHead), vp, i64, i64, vp, vp, sz, vp]
         L.pafu_score_qkv.restype = i32
@@ -212,6 +214,13 @@ def pafu_workspace_bytes(shape: Shape, policy=None, head: Optional[Head] = None)
 
 def pafu_workspace_status(ws: torch.Tensor) -> int:
     return lib().pafu_workspace_status(_ptr(ws), _stream())
+
+
+def pafu_workspace_counters(ws: torch.Tensor) -> np.ndarray:
+    """(exact passes on first/ragged tiles, exact passes forced by a row sum, rescales)."""
+    out = np.zeros(3, dtype=np.int64)
+    _check(lib().pafu_workspace_counters(_ptr(ws), _ptr(out), _stream()), "pafu_workspace_counters")
+    return out
 
 
 def pafu_score(head: Head, X: torch.Tensor, scores: torch.Tensor, ws: Optional[torch.Tensor] = None,

@@ -9,6 +9,12 @@ namespace pafu {
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// true when the byte ranges [a, a + na) and [b, b + nb) share a byte
+static bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb) {
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return na > 0 && nb > 0 && a0 < b0 + nb && b0 < a0 + na;
+}
+
 static bool prefix_ok(const int64_t* cu, int n) {
     if (cu == nullptr || cu[0] != 0) return false;
     for (int s = 0; s < n; ++s)
@@ -52,13 +58,14 @@ static void fill_prefix(int64_t* dst, const int64_t* src, int n) {
     for (int s = 0; s <= n; ++s) dst[s] = src ? src[s] : 0;
 }
 
-static pafu_status head_ok(const pafu_head* h) {
+// `device_ptrs`: the weight pointers are device pointers and must be 16-byte aligned
+static pafu_status head_ok(const pafu_head* h, bool device_ptrs = true) {
     if (h == nullptr || h->w1 == nullptr || h->w2 == nullptr) return PAFU_ERR_INVALID_ARG;
     if (h->d_in < 1 || h->d_hidden < 1 || h->d_out < 1) return PAFU_ERR_INVALID_ARG;
     if (h->act != PAFU_ACT_GELU && h->act != PAFU_ACT_SILU) return PAFU_ERR_INVALID_ARG;
     if (h->final != PAFU_FINAL_NONE && h->final != PAFU_FINAL_SIGMOID) return PAFU_ERR_INVALID_ARG;
     if (h->d_in % 64 != 0 || h->d_hidden % 16 != 0 || h->d_hidden > 1024) return PAFU_ERR_UNSUPPORTED_SHAPE;
-    if (!aligned16(h->w1) || !aligned16(h->w2)) return PAFU_ERR_MISALIGNED;
+    if (device_ptrs && (!aligned16(h->w1) || !aligned16(h->w2))) return PAFU_ERR_MISALIGNED;
     return PAFU_OK;
 }
 
@@ -132,6 +139,19 @@ pafu_status pafu_workspace_status(const void* ws, void* stream) {
     return word == 0 ? PAFU_OK : PAFU_ERR_TIMEOUT;
 }
 
+pafu_status pafu_workspace_counters(const void* ws, int64_t* counts, void* stream) {
+    if (ws == nullptr || counts == nullptr) return PAFU_ERR_INVALID_ARG;
+    int32_t words[3] = {0, 0, 0};
+    static_assert(kStatusWordFullSum == kStatusWordFullFirst + 1 && kStatusWordRescale == kStatusWordFullFirst + 2,
+                  "the three counters are read with one copy");
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(words, static_cast<const int32_t*>(ws) + kStatusWordFullFirst, sizeof words,
+                        cudaMemcpyDeviceToHost, cs) != cudaSuccess) return PAFU_ERR_CUDA;
+    if (cudaStreamSynchronize(cs) != cudaSuccess) return PAFU_ERR_CUDA;
+    for (int i = 0; i < 3; ++i) counts[i] = words[i];
+    return PAFU_OK;
+}
+
 namespace {
 // shared by the one- and three-matrix entry points; X[i] holds features [i * d_in / n_parts, ...)
 pafu_status score_impl(const pafu_head* head, const uint16_t* const* X, int n_parts, int64_t n_tokens, int64_t ldx,
@@ -202,7 +222,13 @@ pafu_status pafu_compact(const uint16_t* K, const uint16_t* V, const float* SL, 
     if (K == nullptr || V == nullptr || idx == nullptr || Kc == nullptr || Vc == nullptr) return PAFU_ERR_INVALID_ARG;
     if ((SL == nullptr) != (SLc == nullptr)) return PAFU_ERR_INVALID_ARG;
     if (!aligned16(K) || !aligned16(V) || !aligned16(Kc) || !aligned16(Vc) || !aligned16(idx)) return PAFU_ERR_MISALIGNED;
-    if (Kc == K || Vc == V || Kc == V || Vc == K) return PAFU_ERR_INVALID_ARG;
+    {
+        const size_t in_b = (size_t)st.cu_T[st.n_streams] * dm * 2, out_b = (size_t)st.cu_B[st.n_streams] * dm * 2;
+        if (ranges_overlap(Kc, out_b, K, in_b) || ranges_overlap(Kc, out_b, V, in_b) || ranges_overlap(Vc, out_b, K, in_b) ||
+            ranges_overlap(Vc, out_b, V, in_b) || ranges_overlap(Kc, out_b, Vc, out_b)) return PAFU_ERR_INVALID_ARG;
+        if (SLc != nullptr && ranges_overlap(SLc, (size_t)st.cu_B[st.n_streams] * 4, SL, (size_t)st.cu_T[st.n_streams] * 4))
+            return PAFU_ERR_INVALID_ARG;
+    }
     return launch_compact(K, V, SL, idx, st, (int32_t)dm, Kc, Vc, SLc, static_cast<cudaStream_t>(stream));
 }
 
@@ -229,7 +255,20 @@ pafu_status pafu_compact_layers(const uint16_t* const* K, const uint16_t* const*
     for (int l = 0; l < n_layers; ++l) {
         if (K[l] == nullptr || V[l] == nullptr || Kc[l] == nullptr || Vc[l] == nullptr) return PAFU_ERR_INVALID_ARG;
         if (!aligned16(K[l]) || !aligned16(V[l]) || !aligned16(Kc[l]) || !aligned16(Vc[l])) return PAFU_ERR_MISALIGNED;
-        if (Kc[l] == K[l] || Vc[l] == V[l] || Kc[l] == V[l] || Vc[l] == K[l]) return PAFU_ERR_INVALID_ARG;
+    }
+    {
+        // no output may overlap any layer's input or another output
+        const size_t in_b = (size_t)st.cu_T[st.n_streams] * dm * 2, out_b = (size_t)st.cu_B[st.n_streams] * dm * 2;
+        for (int l = 0; l < n_layers; ++l) {
+            const void* outs[2] = {Kc[l], Vc[l]};
+            for (const void* o : outs) {
+                for (int m = 0; m < n_layers; ++m) {
+                    if (ranges_overlap(o, out_b, K[m], in_b) || ranges_overlap(o, out_b, V[m], in_b)) return PAFU_ERR_INVALID_ARG;
+                    if (m != l && (ranges_overlap(o, out_b, Kc[m], out_b) || ranges_overlap(o, out_b, Vc[m], out_b))) return PAFU_ERR_INVALID_ARG;
+                }
+            }
+            if (ranges_overlap(Kc[l], out_b, Vc[l], out_b)) return PAFU_ERR_INVALID_ARG;
+        }
     }
     return launch_compact_layers(K, V, n_layers, SL, idx, st, (int32_t)dm, Kc, Vc, SLc, static_cast<cudaStream_t>(stream));
 }
@@ -377,7 +416,13 @@ static pafu_status step_impl(const pafu_step_args* a, void* const* ev, void* str
     const void* ptrs[] = {a->K, a->V, a->Q, a->Kq, a->Vq, a->scores, a->idx, a->Kc, a->Vc, a->SLc, a->O, a->LSE};
     for (const void* p : ptrs)
         if (!aligned16(p)) return PAFU_ERR_MISALIGNED;
-    if (nB > 0 && (a->Kc == a->K || a->Vc == a->V || a->Kc == a->V || a->Vc == a->K)) return PAFU_ERR_INVALID_ARG;
+    {
+        const size_t in_b = (size_t)nT * dm * 2, out_b = (size_t)nB * dm * 2;
+        if (ranges_overlap(a->Kc, out_b, a->K, in_b) || ranges_overlap(a->Kc, out_b, a->V, in_b) ||
+            ranges_overlap(a->Vc, out_b, a->K, in_b) || ranges_overlap(a->Vc, out_b, a->V, in_b) ||
+            ranges_overlap(a->Kc, out_b, a->Vc, out_b)) return PAFU_ERR_INVALID_ARG;
+        if (a->SLc != nullptr && ranges_overlap(a->SLc, (size_t)nB * 4, a->scores, (size_t)nT * 4)) return PAFU_ERR_INVALID_ARG;
+    }
     const size_t need = pafu_workspace_bytes(&a->shape, a->policy, a->head);
     if (a->ws == nullptr) return PAFU_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(a->ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
@@ -390,12 +435,27 @@ static pafu_status step_impl(const pafu_step_args* a, void* const* ev, void* str
     e = pafu_score(a->head, a->K, nT, dm, a->scores, a->ws, a->ws_bytes, stream);
     if (e != PAFU_OK) return e;
     if (!mark(1)) return PAFU_ERR_CUDA;
-    e = pafu_select(a->scores, &a->shape, a->policy, a->idx, a->ws, a->ws_bytes, stream);
+    StreamTable st;
+    memset(&st, 0, sizeof st);
+    st.n_streams = n;
+    fill_prefix(st.cu_T, a->shape.cu_T, n);
+    e = fill_policy(&a->shape, a->policy, &st);
     if (e != PAFU_OK) return e;
-    if (!mark(2)) return PAFU_ERR_CUDA;
-    e = pafu_compact(a->K, a->V, a->SLc ? a->scores : nullptr, a->idx, &a->shape, a->policy, a->Kc, a->Vc,
-                     a->SLc, stream);
-    if (e != PAFU_OK) return e;
+    if (nB > 0 && dm % 8 == 0 && select_compact_fusable(st)) {
+        // Top-k and Select(KV; ids) as one launch: every CTA finds the threshold by itself, then
+        // writes and copies its own share of the kept rows
+        if (!mark(2)) return PAFU_ERR_CUDA;
+        e = launch_select_compact(a->scores, st, a->idx, a->K, a->V, a->SLc ? a->scores : nullptr, (int32_t)dm, a->Kc,
+                                  a->Vc, a->SLc, cs);
+        if (e != PAFU_OK) return e;
+    } else {
+        e = pafu_select(a->scores, &a->shape, a->policy, a->idx, a->ws, a->ws_bytes, stream);
+        if (e != PAFU_OK) return e;
+        if (!mark(2)) return PAFU_ERR_CUDA;
+        e = pafu_compact(a->K, a->V, a->SLc ? a->scores : nullptr, a->idx, &a->shape, a->policy, a->Kc, a->Vc,
+                         a->SLc, stream);
+        if (e != PAFU_OK) return e;
+    }
     if (!mark(3)) return PAFU_ERR_CUDA;
     e = pafu_chunk_attn(a->Q, a->Kc, a->Vc, cu_B, a->Kq, a->Vq, &a->shape, a->scale, a->O, a->LSE,
                         a->ws, a->ws_bytes, stream);
@@ -456,7 +516,12 @@ pafu_status pafu_step_host(const pafu_step_args* a, void* arena, size_t arena_by
     e = pafu_kept_counts(&a->shape, a->policy, cu_B);
     if (e != PAFU_OK) return e;
     const pafu_head* h = a->head;
-    if (h->d_in < 1 || h->d_hidden < 1 || h->d_out < 1 || h->w1 == nullptr || h->w2 == nullptr) return PAFU_ERR_INVALID_ARG;
+    // everything pafu_step would reject is rejected here, before the first copy is enqueued
+    e = head_ok(h, /*device_ptrs=*/false);
+    if (e != PAFU_OK) return e;
+    if (h->d_in != (int64_t)a->shape.n_heads * a->shape.d_head) return PAFU_ERR_INVALID_ARG;
+    if (a->shape.d_head != 64 && a->shape.d_head != 128) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    if (!(a->scale >= 0.f) || isinf(a->scale)) return PAFU_ERR_INVALID_ARG;
     const size_t total = pafu_step_host_arena_bytes(&a->shape, a->policy, h);
     if (total == 0) return PAFU_ERR_INVALID_ARG;
     if (arena_bytes < total) return PAFU_ERR_WORKSPACE_TOO_SMALL;

@@ -58,8 +58,7 @@ constexpr int kNoAllocCtas = 31;
 constexpr size_t kNoAllocBytes = pafu::kWsHeaderBytes + (size_t)kNoAllocCtas * 2 * pafu::attn_tc::kPieceBytes;
 static_assert(kNoAllocBytes <= (size_t)PAFU_NOALLOC_SCRATCH_BYTES, "scratch array too small");
 static __device__ __align__(256) unsigned char g_noalloc_scratch[PAFU_NOALLOC_SCRATCH_BYTES];
-constexpr int kMaxDevices = 64;
-void* g_noalloc_ptr[kMaxDevices] = {nullptr};   // device address of the array, per device
+void* g_noalloc_ptr[pafu::kMaxDevices] = {nullptr};   // device address of the array, per device
 }  // namespace
 
 extern "C" pafu_status pafu_chunk_attn_noalloc(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
@@ -94,7 +93,7 @@ extern "C" pafu_status pafu_chunk_attn_noalloc(const uint16_t* Q, const uint16_t
     // set-up, once per device: in host code the array's name is only a handle, the address the
     // kernels need comes from the runtime
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PAFU_ERR_CUDA;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= pafu::kMaxDevices) return PAFU_ERR_CUDA;
     if (g_noalloc_ptr[dev] == nullptr) {
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return PAFU_ERR_CUDA;

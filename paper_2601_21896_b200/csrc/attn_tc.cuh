@@ -357,7 +357,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 }
             }
             cp_async_wait_all();
-        } else if (elect_one()) {
+        } else if (elect_one() && p.status[kStatusWordStallLoader] == 0) {
             prefetch_tmap(&mQ); prefetch_tmap(&mKc); prefetch_tmap(&mVc);
             if (p.has_chunk) { prefetch_tmap(&mKq); prefetch_tmap(&mVq); }
             SegIter iter(p, blockIdx.x, gridDim.x);
@@ -570,6 +570,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                         if (c >= left) sr[c] = 0xff800000u;   // -inf
                 }
                 if (full_pass) {
+                    if ((tid & 31) == 0) atomicAdd(p.status + ((i == 0 || left < kBN) ? kStatusWordFullFirst : kStatusWordFullSum), 1);
                     float mx4[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
@@ -591,6 +592,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                                                   : mbar_wait(pv_done(slot), pvcnt & 1u)) && !abort_flag;
                         if (!__all_sync(0xffffffffu, w)) { fail(303); ok = false; break; }
                         tc_fence_after_sync();
+                        if ((tid & 31) == 0) atomicAdd(p.status + kStatusWordRescale, 1);
                         const float m_new = fmaxf(m_used, mx);
                         const float alpha = fast_exp2((m_used - m_new) * sl2);
                         l_sum *= alpha;
@@ -850,13 +852,12 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t*
     Params p;
     p.st = st; p.n_heads = n_heads; p.has_chunk = has_chunk; p.scale = scale;
     p.O = O; p.LSE = LSE; p.status = status; p.pieces = pieces; p.idx = idx; p.Kraw = gather ? Kc : nullptr; p.Vraw = gather ? Vc : nullptr; p.total_Lq = nQ; p.total_cost = cost;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-            return PAFU_ERR_CUDA;
-        attr_set = true;
-    }
+    static bool attr_set[kMaxDevices] = {};
+    if (!once_per_device(attr_set, [] {
+            return cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess &&
+                   cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess;
+        }))
+        return PAFU_ERR_CUDA;
     int grid = grid_for(cost);
     if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;   // caller's scratch holds fewer partials
     if ((gather ? launch_dependent(attn_tc_kernel<true>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mKc, mVc, mKq, mVq, p)

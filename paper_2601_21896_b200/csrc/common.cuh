@@ -22,6 +22,13 @@ struct StreamTable {
 // Workspace layout: [0, 256) status header (int32 words), then per-step scratch.
 constexpr size_t kWsHeaderBytes = 256;
 constexpr int kStatusWordTimeout = 0;   // non-zero: a bounded wait ran out
+// Diagnostic counters of the tcgen05 attention kernel, one count per (softmax warp, key tile):
+constexpr int kStatusWordFullFirst = 8;    // exact pass on a run's first tile or a segment's ragged last tile
+constexpr int kStatusWordFullSum = 9;      // exact pass forced by a row sum that outgrew the running maximum
+constexpr int kStatusWordRescale = 10;     // output accumulator and row sum rescaled in tensor memory
+// Test hook: while this word is non-zero the attention kernel's loader role issues no copies, so
+// every consumer's bounded wait runs out and the kernel unwinds with PAFU_ERR_TIMEOUT.
+constexpr int kStatusWordStallLoader = 32;
 
 inline pafu_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? PAFU_OK : PAFU_ERR_CUDA; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -29,17 +36,36 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // SM count of the current device (148 when no device is visible, e.g. sizing queries on a
 // build host); capped so per-CTA tables stay small.
 constexpr int kMaxPersistentGrid = 256;
+constexpr int kMaxDevices = 64;       // per-device caches below are indexed by the CUDA device ordinal
+inline int current_device() {
+    int dev = 0;
+    return (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < kMaxDevices) ? dev : -1;
+}
 inline int device_sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-            n = v < kMaxPersistentGrid ? v : kMaxPersistentGrid;
+    static int n[kMaxDevices] = {};
+    const int dev = current_device();
+    if (dev < 0) return 148;
+    if (n[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n[dev] = v < kMaxPersistentGrid ? v : kMaxPersistentGrid;
         else
             return 148;
     }
-    return n;
+    return n[dev];
+}
+// Runs `set` (the cudaFuncSetAttribute calls of one kernel family) once per device; `done` is
+// that family's per-device record.  Function attributes belong to the device's context, so a
+// process that uses several GPUs has to opt in on each of them.
+template <typename Set>
+inline bool once_per_device(bool (&done)[kMaxDevices], Set set) {
+    const int dev = current_device();
+    if (dev < 0) return false;
+    if (!done[dev]) {
+        if (!set()) return false;
+        done[dev] = true;
+    }
+    return true;
 }
 
 // Every kernel of this library is launched with programmatic stream serialization: its CTAs
@@ -80,6 +106,10 @@ pafu_status launch_score(const pafu_head& head, const uint16_t* const* X, int n_
                          float* scores, void* ws, size_t ws_bytes, cudaStream_t stream);
 pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* idx,
                           cudaStream_t stream);
+bool select_compact_fusable(const StreamTable& st);
+pafu_status launch_select_compact(const float* scores, const StreamTable& st, int32_t* idx, const uint16_t* K,
+                                  const uint16_t* V, const float* SL, int32_t d_model, uint16_t* Kc, uint16_t* Vc,
+                                  float* SLc, cudaStream_t stream);
 pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL,
                            const int32_t* idx, const StreamTable& st, int32_t d_model,
                            uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream);

@@ -96,7 +96,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
     auto empty = [&](int st) { return bar0 + 8 * (kStages + st); };
     auto acc_full = [&](int b) { return bar0 + 8 * (2 * kStages + b); };
     auto acc_empty = [&](int b) { return bar0 + 8 * (2 * kStages + 2 + b); };
-    const uint32_t halves_bar = bar0 + 8 * (2 * kStages + 4);   // column-half 1 -> column-half 0
+    // column-half 1 -> column-half 0, one barrier per half_sum slot: with a single barrier the half-1
+    // warps could complete two tiles' arrivals while a half-0 warp still waits for the first
+    auto halves_bar = [&](int slot) { return bar0 + 8 * (2 * kStages + 4 + slot); };
     __shared__ uint32_t tmem_base_sh;
     __shared__ volatile int abort_flag;
 
@@ -113,7 +115,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
     if (tid == 0) {
         for (int st = 0; st < kStages; ++st) { mbar_init(full(st), 1); mbar_init(empty(st), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full(b), 1); mbar_init(acc_empty(b), 8); }
-        mbar_init(halves_bar, 4);
+        mbar_init(halves_bar(0), 4); mbar_init(halves_bar(1), 4);
         abort_flag = 0;
         fence_barrier_init();
     }
@@ -226,7 +228,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
                 }
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(acc_empty(buf));
+                // the column-half-0 warps hand back a tile's last accumulator only after they have
+                // taken the other half's partial sums (below): the MMAs that reuse the accumulator, and
+                // with them the half-1 warps, can then never run two tiles ahead of a half-0 warp
+                if (lane == 0 && (half == 1 || ch + 1 < ch1)) mbar_arrive(acc_empty(buf));
             }
             if (!ok) break;
             // combine the two column halves of each row
@@ -234,16 +239,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
             if (half == 1) {
                 hs[row] = part;
                 __syncwarp();
-                if (lane == 0) mbar_arrive(halves_bar);
+                if (lane == 0) mbar_arrive(halves_bar(tile_it & 1));
             } else {
-                const bool w = mbar_wait(halves_bar, tile_it & 1u) && !abort_flag;
+                const bool w = mbar_wait(halves_bar(tile_it & 1), (tile_it >> 1) & 1u) && !abort_flag;
                 if (!__all_sync(0xffffffffu, w)) { fail(405); ok = false; break; }
+                const float other = hs[row];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty((acc_it - 1) & 1));
                 const int64_t t = tile * kBM + row;
                 if (p.split) {
                     // this chunk's row sums go to the cluster's first CTA
-                    cooperative_groups::this_cluster().map_shared_rank(chunk_sum, 0)[ch0 * kBM + row] = part + hs[row];
+                    cooperative_groups::this_cluster().map_shared_rank(chunk_sum, 0)[ch0 * kBM + row] = part + other;
                 } else if (t < p.n_tokens) {
-                    float v = part + hs[row] + b2m;
+                    float v = part + other + b2m;
                     if (p.final == PAFU_FINAL_SIGMOID) v = rcpf(1.0f + ex2f(-v * 1.4426950408889634f));
                     p.scores[t] = v;
                 }
@@ -291,13 +299,12 @@ inline pafu_status launch(const pafu_head& head, const uint16_t* const* X, int n
     p.split = (n_chunks > 1 && n_tiles * n_chunks <= 2 * (int64_t)sm_count) ? 1 : 0;
     const int grid = p.split ? (int)(n_tiles * n_chunks) : (int)(n_tiles < sm_count ? n_tiles : sm_count);
     const unsigned cluster = p.split ? (unsigned)n_chunks : 1u;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(score_tc_kernel<PAFU_ACT_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(score_tc_kernel<PAFU_ACT_SILU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-            return PAFU_ERR_CUDA;
-        attr_set = true;
-    }
+    static bool attr_set[kMaxDevices] = {};
+    if (!once_per_device(attr_set, [] {
+            return cudaFuncSetAttribute(score_tc_kernel<PAFU_ACT_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess &&
+                   cudaFuncSetAttribute(score_tc_kernel<PAFU_ACT_SILU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess;
+        }))
+        return PAFU_ERR_CUDA;
     return cuda_ok(head.act == PAFU_ACT_GELU
                        ? launch_dependent(score_tc_kernel<PAFU_ACT_GELU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, cluster, mX[0], mX[1], mX[2], mW, p)
                        : launch_dependent(score_tc_kernel<PAFU_ACT_SILU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, cluster, mX[0], mX[1], mX[2], mW, p));

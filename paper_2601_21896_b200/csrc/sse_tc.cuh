@@ -432,13 +432,12 @@ inline pafu_status launch(const uint16_t* Q, const uint16_t* K, const float* lse
     CUtensorMap mQ, mK;
     if (!TmapEncoder::token_tensor(&mQ, Q, (uint64_t)L, n_heads, kD, kBT) ||
         !TmapEncoder::token_tensor(&mK, K, (uint64_t)L, n_heads, kD, kBT)) return PAFU_ERR_CUDA;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(sse_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
-            cudaFuncSetAttribute(sse_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-            return PAFU_ERR_CUDA;
-        attr_set = true;
-    }
+    static bool attr_set[kMaxDevices] = {};
+    if (!once_per_device(attr_set, [] {
+            return cudaFuncSetAttribute(sse_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess &&
+                   cudaFuncSetAttribute(sse_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess;
+        }))
+        return PAFU_ERR_CUDA;
     const int sms = device_sm_count();
     const int64_t n_pad = (int64_t)n_heads * p.n_qt * (kAugBytes / 2);
     const int g0 = (int)((n_pad + 255) / 256 < 8 * sms ? (n_pad + 255) / 256 : 8 * sms);

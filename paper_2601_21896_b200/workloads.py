@@ -268,3 +268,72 @@ def sample_rows(n_rows: int, n_sample: int, seed: int = 0, tile: int = 128, tag:
     rest = rng.choice(n_rows, size=n_sample, replace=False)
     rows = np.array(sorted(must | set(int(r) for r in rest[: n_sample - len(must)])), dtype=np.int64)
     return rows
+
+
+def peaked_attention_inputs(kind: str, n_heads: int, d_head: int, Lq: int, nB: int, seed: int = 0,
+                            q_scale: float = 1.0, rise_per_tile: float = 0.0, spike_pos: Sequence[int] = (),
+                            spike_gain: float = 4.0, varied_rows: bool = False, tile: int = 64,
+                            tiny_every: int = 3, tiny_gain: float = 5.0) -> Dict[str, np.ndarray]:
+    """Inputs whose attention rows are NOT near-uniform (real attention maps are peaked: Sec. 3.2),
+    so that a tiled softmax has to move its running maximum.  Returns bf16 bit patterns
+    Q [Lq, N, D], Kc/Vc [nB, N, D] (retained segment), Kq/Vq [Lq, N, D] (chunk segment); keys are
+    numbered retained first, then chunk.  Every query carries a component g_i along the all-ones
+    direction e and key j a component a_j, so logit(i, j) ~ a_j (g_i sqrt(D) + xi_i) + N(0, ~1):
+
+      "scaled_q"    plain Gaussian Q, K with Q multiplied by q_scale (logit spread q_scale nats)
+      "ramp"        a_j rises linearly along the key axis by rise_per_tile nats per 64 keys
+                    (negative: falls), so the row maximum moves in every tile (or never)
+      "spike"       keys at positions spike_pos are spike_gain * e: each dominates its row by
+                    ~spike_gain * sqrt(D) nats; the k-th listed spike is (1 + k/2) times stronger,
+                    so later ones overtake earlier ones
+      "tiny_tiles"  every tiny_every-th 64-key tile of each segment is pushed ~tiny_gain * sqrt(D)
+                    nats below the rest: a run that opens on such a tile starts from a far too
+                    small maximum
+    varied_rows draws g_i uniformly from [-1, 2] instead of 1: in one 32-row group some rows
+    see the spike as dominant, some as negligible, some not at all.
+    """
+    N, D = n_heads, d_head
+    rq = rng_for(seed, 97, 0, 0, "Q"); rk = rng_for(seed, 97, 0, 0, "K"); rv = rng_for(seed, 97, 0, 0, "V")
+    Q = _normal(rq, (Lq, N, D)); K = _normal(rk, (nB + Lq, N, D)); V = _normal(rv, (nB + Lq, N, D))
+    root = np.float32(np.sqrt(D))
+    if kind == "scaled_q":
+        Q *= np.float32(q_scale)
+    else:
+        g = np.ones((Lq, 1, 1), np.float32)
+        if varied_rows:
+            g = rng_for(seed, 97, 0, 0, "misc").uniform(-1.0, 2.0, size=(Lq, 1, 1)).astype(np.float32)
+        Q += g
+        if kind == "ramp":
+            j = np.arange(nB + Lq, dtype=np.float32).reshape(-1, 1, 1)
+            K += np.float32(rise_per_tile) * (j / np.float32(tile)) / root
+        elif kind == "spike":
+            for k, pos in enumerate(spike_pos):
+                K[pos] = np.float32(spike_gain * (1.0 + 0.5 * k))
+        elif kind == "tiny_tiles":
+            for lo, hi in ((0, nB), (nB, nB + Lq)):
+                for t0 in range(lo, hi, tile * tiny_every):
+                    K[t0:min(t0 + tile, hi)] -= np.float32(tiny_gain)
+        else:
+            raise KeyError(kind)
+    b = f32_to_bf16_bits
+    return {"Q": b(Q), "Kc": b(K[:nB]), "Vc": b(V[:nB]), "Kq": b(K[nB:]), "Vq": b(V[nB:])}
+
+
+def queries_from_keys(w: Workload, d: Dict[str, np.ndarray], seed: int = 0) -> np.ndarray:
+    """Replacement for d["Q"]: query i of a stream is a copy (all heads) of one key row the
+    retention rule always keeps - a sink or recent row of the cache - or of one of the chunk's own
+    key rows, alternating.  q = k makes that key's logit |k|^2 / sqrt(D) ~ 14 nats at these
+    input statistics against ~1.3 nats of spread for the others: peaked attention rows."""
+    cuT, cuQ = w.cu("T"), w.cu("Lq")
+    out = d["Q"].copy()
+    for s in range(w.n_streams):
+        rng = rng_for(seed, 96, 0, s, "Q")
+        T, Lq, B = w.T[s], w.Lq[s], min(w.budget[s], w.T[s])
+        nr = min(w.n_recent, B); ns = min(w.n_sink, B - nr)
+        always = np.concatenate([np.arange(ns), np.arange(T - nr, T)]) if T > B else np.arange(T)
+        for i in range(Lq):
+            if (i & 1) and len(always):
+                out[cuQ[s] + i] = d["K"][cuT[s] + always[rng.integers(len(always))]]
+            else:
+                out[cuQ[s] + i] = d["Kq"][cuQ[s] + rng.integers(Lq)]
+    return out

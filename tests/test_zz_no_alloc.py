@@ -15,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2601_21896_b200 as pafu
 from paper_2601_21896_b200 import workloads as wl
 from paper_2601_21896_b200.harness import Layer, bf16_to_bits
@@ -35,6 +36,13 @@ def test_noalloc_matches_workspace_entry_point_twice():
         L.score(); L.select(); L.compact()
         L.attn(); L.check_status()
         want_O, want_lse = _as_f32(L.O), L.LSE.cpu().numpy().astype(np.float64)
+        truth = None
+        if w.name == "small_ragged":
+            # small enough for the CPU oracle: compare with the definition as well, stream by stream
+            Kc, Vc = bf16_to_bits(L.Kc), bf16_to_bits(L.Vc)
+            cuB, cuQ = L.cu_B, w.cu("Lq")
+            truth = [oracle.attention(d["Q"][cuQ[s]:cuQ[s + 1]], Kc[cuB[s]:cuB[s + 1]], Vc[cuB[s]:cuB[s + 1]],
+                                      d["Kq"][cuQ[s]:cuQ[s + 1]], d["Vq"][cuQ[s]:cuQ[s + 1]]) for s in range(w.n_streams)]
         for call in range(2):
             O = torch.full_like(L.O, float("nan"))
             LSE = torch.full_like(L.LSE, float("nan"))
@@ -46,6 +54,11 @@ def test_noalloc_matches_workspace_entry_point_twice():
             assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (w.name, call, err.max(), err.mean())
             err = np.abs(got_lse - want_lse)
             assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (w.name, call, err.max())
+            if truth is not None:
+                for s, (tO, tL) in enumerate(truth):
+                    err = np.abs(got_O[cuQ[s]:cuQ[s + 1]] - tO)
+                    assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, ("oracle", s, call, err.max(), err.mean())
+                    assert np.abs(got_lse[:, cuQ[s]:cuQ[s + 1]] - tL).max() <= MAX_ABS, ("oracle LSE", s, call)
 
 
 @pytest.mark.gpu
