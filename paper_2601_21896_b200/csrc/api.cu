@@ -441,12 +441,16 @@ static pafu_status step_impl(const pafu_step_args* a, void* const* ev, void* str
     fill_prefix(st.cu_T, a->shape.cu_T, n);
     e = fill_policy(&a->shape, a->policy, &st);
     if (e != PAFU_OK) return e;
-    if (nB > 0 && dm % 8 == 0 && select_compact_fusable(st)) {
-        // Top-k and Select(KV; ids) as one launch: every CTA finds the threshold by itself, then
-        // writes and copies its own share of the kept rows
+    if (nB > 0 && dm % 8 == 0) {
+        // Top-k and Select(KV; ids) overlapped: the gather is launched as a programmatic dependent of
+        // the selection, copies the always-kept rows while the selection runs and the top-k rows
+        // once the indices exist.  No event may sit between the two launches, so in the timed
+        // variant the "after select" stamp is taken before them.
         if (!mark(2)) return PAFU_ERR_CUDA;
-        e = launch_select_compact(a->scores, st, a->idx, a->K, a->V, a->SLc ? a->scores : nullptr, (int32_t)dm, a->Kc,
-                                  a->Vc, a->SLc, cs);
+        e = launch_select(a->scores, st, a->idx, cs);
+        if (e != PAFU_OK) return e;
+        e = launch_compact(a->K, a->V, a->SLc ? a->scores : nullptr, a->idx, st, (int32_t)dm, a->Kc, a->Vc, a->SLc, cs,
+                           /*always_first=*/true);
         if (e != PAFU_OK) return e;
     } else {
         e = pafu_select(a->scores, &a->shape, a->policy, a->idx, a->ws, a->ws_bytes, stream);

@@ -77,6 +77,9 @@ inline bool once_per_device(bool (&done)[kMaxDevices], Set set) {
 // bandwidth-bound kernel was still in its last wave cost more than the earlier start gained.
 #ifdef __CUDACC__
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the kernel launched behind this one (as a programmatic dependent) start now; that kernel
+// still sees this one's results only after its own grid_dep_wait().
+__device__ __forceinline__ void grid_dep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
@@ -106,13 +109,11 @@ pafu_status launch_score(const pafu_head& head, const uint16_t* const* X, int n_
                          float* scores, void* ws, size_t ws_bytes, cudaStream_t stream);
 pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* idx,
                           cudaStream_t stream);
-bool select_compact_fusable(const StreamTable& st);
-pafu_status launch_select_compact(const float* scores, const StreamTable& st, int32_t* idx, const uint16_t* K,
-                                  const uint16_t* V, const float* SL, int32_t d_model, uint16_t* Kc, uint16_t* Vc,
-                                  float* SLc, cudaStream_t stream);
+// always_first: the rows that are kept whatever the scores say are copied before the kernel waits
+// for its predecessor (only valid when that predecessor is launch_select of the same step)
 pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL,
                            const int32_t* idx, const StreamTable& st, int32_t d_model,
-                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream);
+                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream, bool always_first = false);
 pafu_status launch_compact_layers(const uint16_t* const* K, const uint16_t* const* V, int32_t n_layers,
                                   const float* SL, const int32_t* idx, const StreamTable& st, int32_t d_model,
                                   uint16_t* const* Kc, uint16_t* const* Vc, float* SLc, cudaStream_t stream);

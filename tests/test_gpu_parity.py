@@ -14,13 +14,18 @@ pytestmark = pytest.mark.gpu
 
 MAX_ABS, MEAN_ABS = 2e-2, 2e-3
 # Beside the absolute bounds, an error bound relative to the size of the result: bf16 rounding of
-# the output alone gives a relative Frobenius error of 2^-9 / sqrt(3) = 1.1e-3, the bf16
-# probabilities about as much again, so 1e-2 leaves room and still rejects a result that is
-# 1 % off when the values themselves are ~0.01 (near-uniform attention over thousands of keys).
-REL_FRO = 1e-2
+# the output alone gives a relative Frobenius error of about 2^-9 / sqrt(3) = 1.1e-3, the bf16
+# probabilities about as much again (2.0e-3 to 2.3e-3 is what the kernels show on every input),
+# so 5e-3 leaves room and still rejects a result that is half a percent off when the values
+# themselves are ~0.01 (near-uniform attention over thousands of keys).
+REL_FRO = 5e-3
 
 
-def close(got, want, what=""):
+def close(got, want, what="", scaled=False):
+    """The benchmark spec's bounds (max-abs 2e-2, mean-abs 2e-3) plus the relative bound above.  `scaled`:
+    the inputs were built to give outputs of magnitude up to ~4.5 (attention that picks single
+    value rows); bf16 rounding of an output o alone is up to 2^-8 |o| = 1.8e-2 there, and the bf16
+    probabilities add up to 2^-8 max|v|, so the absolute bounds grow with max|want|."""
     got = np.asarray(got, dtype=np.float64); want = np.asarray(want, dtype=np.float64)
     assert got.shape == want.shape, (got.shape, want.shape)
     if got.size == 0:
@@ -31,8 +36,9 @@ def close(got, want, what=""):
     rel = np.sqrt((err * err).sum()) / norm if norm > 1e-30 else 0.0
     print("%s: max-abs %.3e mean-abs %.3e rel-fro %.3e (max|want| %.3g)" % (what, err.max(), err.mean(), rel,
                                                                              np.abs(want).max()))
-    assert err.max() <= MAX_ABS, (what, err.max(), np.unravel_index(err.argmax(), err.shape))
-    assert err.mean() <= MEAN_ABS, (what, err.mean())
+    grow = max(1.0, np.abs(want).max()) if scaled else 1.0
+    assert err.max() <= MAX_ABS * grow, (what, err.max(), np.unravel_index(err.argmax(), err.shape))
+    assert err.mean() <= MEAN_ABS * grow, (what, err.mean())
     assert rel <= REL_FRO, (what, rel)
 
 
@@ -249,7 +255,7 @@ def _attention_all_entry_points(d, N, D, Lq, nB, what, seed=0):
                 torch.full((N, Lq), float("nan"), device="cuda"))
 
     def check(O, LSE, name):
-        close(wl.bf16_bits_to_f32(bf16_to_bits(O)), want_O, "%s %s O" % (what, name))
+        close(wl.bf16_bits_to_f32(bf16_to_bits(O)), want_O, "%s %s O" % (what, name), scaled=True)
         close(LSE.cpu().numpy(), want_lse, "%s %s LSE" % (what, name))
 
     O, LSE = fresh()
@@ -646,7 +652,7 @@ def _full_size_check(w, n_rows=256, seed=0, score_rows=None, peaked=False):
     got = wl.bf16_bits_to_f32(bf16_to_bits(L.O))
     lse = L.LSE.cpu().numpy()
     for s, (O, Ls) in enumerate(oracle_attn_streams(w, d, Kc_bits, Vc_bits, cuB, rows)):
-        close(got[cuQ[s]:cuQ[s + 1]][rows[s]], O, "O stream %d" % s)
+        close(got[cuQ[s]:cuQ[s + 1]][rows[s]], O, "O stream %d" % s, scaled=peaked)
         close(lse[:, cuQ[s]:cuQ[s + 1]][:, rows[s]], Ls, "LSE stream %d" % s)
 
 
