@@ -3,14 +3,18 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
-One "step" is one pass of the whole path over one layer's synthetic inputs.  The default
+One "step" is one pass of the whole path over one layer's synthetic inputs.  The headline
 workload is the single Wan-1.3B-class layer: 12 heads x 128, a 28 080-token cache pruned to
 14 040 (1560 sink + 4680 recent + 7800 by salience), 4680 chunk queries.  Prints one JSON line.
 
-`value` is chunk-attention TFLOP/s over the whole step (attention FLOPs / step time, all four
-kernels included) with inputs resident in HBM; `roofline` describes the attention kernel alone;
-`e2e` is the same metric through pafu_step_host with pinned host buffers; `cpu_baseline` is the
-CPU oracle timed on a bounded sample.  `--impl reference` times that oracle instead.
+`value` is chunk-attention TFLOP/s over the whole step (attention FLOPs / step time, all kernels
+included) with inputs resident in HBM; `roofline` describes the attention kernel alone;
+`kernels` splits the step and times each kernel alone with a cold and a warm L2; `e2e` is the
+same metric through pafu_step_host with pinned host buffers; `cpu_baseline` is the CPU oracle
+timed on a bounded sample; `configs` holds the other measured configurations (the 30-layer
+denoising step at three retention budgets, the long-horizon cache, the batch-4 14B-class layer),
+each with its own step time, kernel split, roofline fraction and sampled clocks.
+`--impl reference` times the oracle instead.
 """
 from __future__ import annotations
 
@@ -31,6 +35,8 @@ if ROOT not in sys.path:
 METRIC = "chunk-attn TFLOP/s over salience-pruned KV; ms/denoise step; % of roofline"
 UNIT = "TFLOP/s"
 N_LAYERS_PER_DENOISE_STEP = 30
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}     # vendor figures: HBM3e ~8 TB/s, dense bf16 2.25 PFLOP/s
+SPLIT_ITERS = 50                                           # timed iterations of every per-kernel figure
 
 
 def measured_peaks():
@@ -45,7 +51,7 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples nvidia-smi clocks and throttle reasons while a timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -63,8 +69,10 @@ class ClockSampler:
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
+            time.sleep(0.15)
         except Exception:
             self.proc = None
+        return self
 
     def _read(self):
         for line in self.proc.stdout:
@@ -116,15 +124,15 @@ def recorded_traffic(w):
 
 
 def launches_per_step(w):
-    """Kernels of this library one step launches: score, select (register and/or streaming
+    """Kernels of this library one step launches: score, select (shared-memory and/or streaming
     variant), compact, attention (+ the merge of split items for d_head 128)."""
-    regs = stream = False
+    smem = stream = False
     for t, b in zip(w.T, w.budget):
-        if b < t and t - min(w.n_sink, b) - min(w.n_recent, b) <= 131072:
-            regs = True
-        else:
+        if b < t and t - min(w.n_sink, b) - min(w.n_recent, b) > 90112:
             stream = True
-    return 1 + int(regs) + int(stream) + 1 + (2 if w.d_head == 128 else 1)
+        else:
+            smem = True
+    return 1 + int(smem) + int(stream) + 1 + (2 if w.d_head == 128 else 1)
 
 
 def pick_workload(name: str):
@@ -134,6 +142,16 @@ def pick_workload(name: str):
     if name.startswith("wan1.3b_layer_b"):
         return wl.wan13b_layer(int(name.rsplit("b", 1)[1]) / 100.0)
     return wl.CONFIGS[name]()
+
+
+def make_config(w, n_layers, n_sets):
+    """The `config` object of the JSON line: identical in both arms."""
+    return {"workload": w.name, "heads": w.n_heads, "d_head": w.d_head, "cache_tokens": list(w.T),
+            "budget": list(w.budget), "n_sink": w.n_sink, "n_recent": w.n_recent,
+            "chunk_tokens": list(w.Lq), "head_mlp": [w.d_model, w.d_hidden, w.d_out],
+            "layers_per_step": n_layers,
+            "l2": "inputs larger than L2: %d independent layer buffer sets (>= 300 MB each) used "
+                  "round-robin, no flush" % n_sets}
 
 
 def algorithmic_work(w):
@@ -212,6 +230,8 @@ def run_reference(args):
     w = pick_workload(args.workload)
     steps = args.steps if args.steps is not None else 3
     warmup = args.warmup if args.warmup is not None else 1
+    n_layers = max(1, args.layers)
+    n_sets = max(args.sets, n_layers) if n_layers > 1 else args.sets
     d = wl.make_layer(w)
     probe = oracle_sampled_step(w, d, 256, 8 * w.n_streams)
     per_step_budget = max(0.2, 90.0 / (steps + warmup))
@@ -222,15 +242,14 @@ def run_reference(args):
     est = []
     for _ in range(steps):
         est.append(oracle_sampled_step(w, d, n_tok, n_rows)["full_step_est_s"])
-    ms = 1e3 * float(np.mean(est))
-    value = w.attn_flops() / (ms * 1e-3) / 1e12
+    ms = 1e3 * float(np.mean(est)) * n_layers
+    value = n_layers * w.attn_flops() / (ms * 1e-3) / 1e12
     sample = ("each step: score on %d of %d tokens, select and compact in full, attention on %d of %d "
               "query rows; step time extrapolated to the full workload" % (n_tok, sum(w.T), n_rows, sum(w.Lq)))
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "heads": w.n_heads, "d_head": w.d_head, "cache_tokens": list(w.T),
-                       "budget": list(w.budget), "chunk_tokens": list(w.Lq)},
+            "config": make_config(w, n_layers, n_sets),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -239,6 +258,172 @@ def run_reference(args):
 
 
 # -------------------------------------------------------------------------------------- ours
+class Bench:
+    """Timing helpers shared by the headline and the per-configuration blocks."""
+
+    def __init__(self, local_rank, world, peaks):
+        import torch
+        import paper_2601_21896_b200 as pafu
+        self.torch, self.pafu = torch, pafu
+        self.local, self.world, self.peaks = local_rank, world, peaks
+        self.stream = torch.cuda.current_stream()
+        self.flush = None
+
+    def events(self, n):
+        ev = [self.torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for e in ev:
+            e.record(self.stream)          # torch creates the cudaEvent_t on first record
+        return ev
+
+    def flush_l2(self):
+        if self.flush is None:
+            self.flush = self.torch.empty(256 << 20, dtype=self.torch.uint8, device="cuda")
+            self.n_flush = 0
+        self.n_flush += 1
+        self.flush.fill_(self.n_flush & 1)          # 256 MB written: twice the L2
+
+    @staticmethod
+    def stats(us):
+        us = np.asarray(us, dtype=np.float64)
+        return {"median": float(np.median(us)), "min": float(us.min()), "mean": float(us.mean()), "n": int(us.size)}
+
+    def time_alone(self, fn, sets, mode):
+        """SPLIT_ITERS launches of one kernel, an event pair around each.  mode "cold": 256 MB are
+        written between launches and the buffer sets rotate; "warm": one buffer set, launched
+        again and again.  Returns microseconds."""
+        torch = self.torch
+        for i in range(5):
+            fn(sets[i % len(sets)] if mode == "cold" else sets[0])
+        ev = [self.events(2) for _ in range(SPLIT_ITERS)]
+        torch.cuda.synchronize()
+        for i, (a, b) in enumerate(ev):
+            L = sets[i % len(sets)] if mode == "cold" else sets[0]
+            if mode == "cold":
+                self.flush_l2()
+            a.record(self.stream)
+            fn(L)
+            b.record(self.stream)
+        torch.cuda.synchronize()
+        return self.stats([a.elapsed_time(b) * 1e3 for a, b in ev])
+
+    def time_back_to_back(self, fn, sets):
+        """SPLIT_ITERS launches with nothing between them (each launch's set-up overlaps the end of
+        the one before), buffer sets rotating; microseconds per launch."""
+        for i in range(5):
+            fn(sets[i % len(sets)])
+        a, b = self.events(2)
+        self.torch.cuda.synchronize()
+        a.record(self.stream)
+        for i in range(SPLIT_ITERS):
+            fn(sets[i % len(sets)])
+        b.record(self.stream)
+        self.torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / SPLIT_ITERS
+
+    def measure(self, w, layers, n_sets, n_layers, steps, warmup, sample_clocks=True, alone=True):
+        """Times `steps` steps of `n_layers` layer passes each (pafu_step, nothing else in the timed
+        region), then the split of the step into its kernels and each kernel alone."""
+        import torch.distributed as dist
+        from paper_2601_21896_b200 import sharding
+        torch, pafu = self.torch, self.pafu
+        work = algorithmic_work(w)
+        peaks = self.peaks
+        for i in range(warmup * n_layers):
+            layers[i % n_sets].step()
+        for L in layers:
+            L.check_status()
+        start, end = self.events(2)
+        sampler = ClockSampler(self.local).start() if sample_clocks else None
+        torch.cuda.synchronize()
+        if self.world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t_wall0 = time.time()
+        start.record(self.stream)
+        for i in range(steps * n_layers):
+            layers[i % n_sets].step()
+        end.record(self.stream)
+        torch.cuda.synchronize()
+        if self.world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t_wall1 = time.time()
+        clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+        for L in layers:
+            L.check_status()
+        total_ms = sharding.max_over_ranks(start.elapsed_time(end), device="cuda")
+        ms_per_step = total_ms / steps
+        value = self.world * n_layers * work["attn_flops"] / (ms_per_step * 1e-3) / 1e12
+
+        # ---- the step's kernels, from events recorded inside the step (pafu_step_timed): score,
+        # selection + row gather (two launches that overlap), attention + merge
+        n_it = max(SPLIT_ITERS, n_layers)
+        step_events = [self.events(5) for _ in range(n_it)]
+        handles = [pafu.event_handles(ev) for ev in step_events]
+        torch.cuda.synchronize()
+        for i in range(n_it):
+            pafu.pafu_step_timed(layers[i % n_sets].args, handles[i])
+        torch.cuda.synchronize()
+        parts = np.array([[ev[0].elapsed_time(ev[1]), ev[2].elapsed_time(ev[3]), ev[3].elapsed_time(ev[4])]
+                          for ev in step_events]) * 1e3                       # microseconds
+        sc, sg, at = (self.stats(parts[:, j]) for j in range(3))
+        capped = bool(clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and
+                      clocks["sm_mhz"] < 0.85 * clocks["sm_max_mhz"])
+        burst = total_ms < 1500.0 and not capped
+        peak_tf = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+        gbs = lambda b, us: b / (us * 1e-6) / 1e9
+        attn_tf = work["attn_flops"] / (at["median"] * 1e-6) / 1e12
+        mem_bytes = work["score_bytes"] + work["select_bytes"] + work["compact_bytes"]
+        mem_us = sc["median"] + sg["median"]
+        out = {
+            "workload": w.name, "ms_per_step": ms_per_step, "value": value, "unit": UNIT,
+            "steps": steps, "layers_per_step": n_layers,
+            "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step / n_layers,
+            "roofline": {"kernel": "chunk attention (+ merge of split items)", "bound": "tensor", "achieved": attn_tf,
+                         "peak": peak_tf, "unit": "TFLOP/s", "frac": attn_tf / peak_tf,
+                         "frac_of_burst": attn_tf / peaks["bf16_tflops"],
+                         "frac_of_sustained": attn_tf / peaks["bf16_tflops_sustained"],
+                         "frac_nominal": attn_tf / NOMINAL["bf16_tflops"], "traffic": recorded_traffic(w),
+                         "peak_source": "%s, %s" % (peaks["source"], "burst" if burst else "sustained")},
+            "kernels_in_step": {
+                "how": "CUDA events recorded inside %d steps (pafu_step_timed); microseconds" % n_it,
+                "score": dict(sc, **{"GB/s": gbs(work["score_bytes"], sc["median"]),
+                                     "TFLOP/s": work["score_flops"] / (sc["median"] * 1e-6) / 1e12,
+                                     "hbm_frac": gbs(work["score_bytes"], sc["median"]) / peaks["hbm_gbs"],
+                                     "hbm_frac_nominal": gbs(work["score_bytes"], sc["median"]) / NOMINAL["hbm_gbs"]}),
+                "select+compact": dict(sg, **{"GB/s": gbs(work["select_bytes"] + work["compact_bytes"], sg["median"]),
+                                              "hbm_frac": gbs(work["select_bytes"] + work["compact_bytes"], sg["median"]) / peaks["hbm_gbs"],
+                                              "note": "two launches; the gather copies the always-kept rows while the selection runs"}),
+                "attn": dict(at, **{"TFLOP/s": attn_tf, "tensor_frac": attn_tf / peak_tf}),
+                "score+select+compact": {"us": mem_us, "GB/s": gbs(mem_bytes, mem_us),
+                                         "hbm_frac": gbs(mem_bytes, mem_us) / peaks["hbm_gbs"],
+                                         "hbm_frac_nominal": gbs(mem_bytes, mem_us) / NOMINAL["hbm_gbs"]},
+            },
+            "clocks": clocks,
+        }
+        if alone:
+            sets = layers[:n_sets]
+            ka = {"how": "each kernel launched alone, %d launches, an event pair around each; cold = 256 MB written "
+                         "between launches and rotating buffer sets, warm = one buffer set relaunched, back_to_back "
+                         "= nothing between launches, rotating buffer sets; microseconds" % SPLIT_ITERS}
+            for name, fn, nbytes in (("score", lambda L: L.score(), work["score_bytes"]),
+                                     ("select", lambda L: L.select(), work["select_bytes"]),
+                                     ("compact", lambda L: L.compact(), work["compact_bytes"])):
+                cold, warm = self.time_alone(fn, sets, "cold"), self.time_alone(fn, sets, "warm")
+                b2b = self.time_back_to_back(fn, sets)
+                ka[name] = {"cold": cold, "warm": warm, "back_to_back": b2b,
+                            "GB/s_cold": gbs(nbytes, cold["median"]), "GB/s_back_to_back": gbs(nbytes, b2b),
+                            "hbm_frac_cold": gbs(nbytes, cold["median"]) / peaks["hbm_gbs"],
+                            "hbm_frac_back_to_back": gbs(nbytes, b2b) / peaks["hbm_gbs"],
+                            "hbm_frac_nominal_back_to_back": gbs(nbytes, b2b) / NOMINAL["hbm_gbs"]}
+            cold = self.time_alone(lambda L: L.attn(), sets, "cold")
+            ka["attn"] = {"cold": cold, "TFLOP/s_cold": work["attn_flops"] / (cold["median"] * 1e-6) / 1e12}
+            for L in sets:
+                L.check_status()
+            out["kernels_alone"] = ka
+        return out, total_ms
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -260,6 +445,9 @@ def run_ours(args):
     w = pick_workload(args.workload)
     work = algorithmic_work(w)
     peaks = measured_peaks()
+    B = Bench(local, world, peaks)
+    stream = B.stream
+    new_events = B.events
 
     # independent layer units per rank (weak scaling: no data-path collective)
     n_layers = max(1, args.layers)
@@ -267,51 +455,15 @@ def run_ours(args):
     layers, host0 = [], None
     my_units = sharding.units_for_rank(world * n_sets, rank, world)
     for i, unit in enumerate(my_units):
-        d = wl.make_layer(w, seed=0, layer=unit)
         if i == 0:
-            host0 = d
+            host0 = wl.make_layer(w, seed=0, layer=unit)       # host copy: the e2e leg and the CPU baseline need it
+            d = host0
+        else:
+            d = wl.make_layer_device(w, seed=0, layer=unit)
         layers.append(Layer(w, d, want_lse=False, want_slc=True))
-    stream = torch.cuda.current_stream()
 
-    def new_events(n):
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
-        for e in ev:
-            e.record(stream)          # torch creates the cudaEvent_t on first record
-        return ev
-
-    for i in range(warmup * n_layers):
-        layers[i % n_sets].step()
-    for L in layers:
-        L.check_status()
-    step_events = [new_events(5) for _ in range(steps * n_layers)]
-    handles = [pafu.event_handles(ev) for ev in step_events]
-    start, end = new_events(2)
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.15)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    t_wall0 = time.time()
-    start.record(stream)
-    for i in range(steps * n_layers):
-        pafu.pafu_step_timed(layers[i % n_sets].args, handles[i])
-    end.record(stream)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    t_wall1 = time.time()
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
-    for L in layers:
-        L.check_status()
-    total_ms = sharding.max_over_ranks(start.elapsed_time(end), device="cuda")
-    parts = np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(4)] for ev in step_events])
-    k_ms = parts.mean(axis=0)          # score, select, compact, attn (per layer)
-    ms_per_step = total_ms / steps
-    value = world * n_layers * work["attn_flops"] / (ms_per_step * 1e-3) / 1e12
+    head, total_ms = B.measure(w, layers, n_sets, n_layers, steps, warmup, alone=(rank == 0))
+    ms_per_step, value, clocks = head["ms_per_step"], head["value"], head["clocks"]
 
     # ---- the same step with Select(KV; ids) applied inside the attention loader (no compaction
     # copy): whole steps, then the indexed attention alone on the indices the steps left behind
@@ -327,7 +479,7 @@ def run_ours(args):
         i1.record(stream)
         torch.cuda.synchronize()
         idx_ms = sharding.max_over_ranks(i0.elapsed_time(i1) / steps, device="cuda")
-        ev_a = [new_events(2) for _ in range(min(steps, 50))]
+        ev_a = [new_events(2) for _ in range(SPLIT_ITERS)]
         for i, (a, b) in enumerate(ev_a):
             a.record(stream)
             layers[i % n_sets].attn_indexed()
@@ -335,7 +487,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         for L in layers:
             L.check_status()
-        ia_ms = float(np.mean([a.elapsed_time(b) for a, b in ev_a]))
+        ia_ms = float(np.median([a.elapsed_time(b) for a, b in ev_a]))
         indexed = {"api": "pafu_step_indexed (score, select, attention reading K/V rows through idx)",
                    "ms_per_step": idx_ms,
                    "value": world * n_layers * work["attn_flops"] / (idx_ms * 1e-3) / 1e12, "unit": UNIT,
@@ -403,6 +555,7 @@ def run_ours(args):
     h2d = sum(int(v.numel() * v.element_size()) for v in hin.values())
     d2h = int(h_scores.numel() * 4 + h_idx.numel() * 4 + h_O.numel() * 2)
     e2e_value = world * work["attn_flops"] / (e2e_ms * 1e-3) / 1e12
+    del arena
 
     # ---- the paper's own S-MLP on the new chunk (Appendix A: [q, k, v] -> 1024 -> 12, SiLU, mean),
     # read from the chunk's Q / K / V in place.  Its 43 MB of inputs fit in L2, so a buffer larger
@@ -416,11 +569,10 @@ def run_ours(args):
                           wl.ACT_SILU, wl.FINAL_NONE)
         pws = torch.zeros(pafu.pafu_workspace_bytes(L0.shape, None, phead), dtype=torch.uint8, device="cuda")
         pout = torch.empty(L0.nQ, dtype=torch.float32, device="cuda")
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         reps = 12
         evq = [new_events(2) for _ in range(reps)]
         for r in range(reps + 3):
-            flush.fill_(r & 1)
+            B.flush_l2()
             if r >= 3:
                 evq[r - 3][0].record(stream)
             pafu.pafu_score_qkv(phead, L0.Q, L0.Kq, L0.Vq, pout, pws, n_tokens=L0.nQ, ld=w.d_model)
@@ -434,7 +586,6 @@ def run_ours(args):
         qkv = {"workload": "paper S-MLP on the chunk: %d tokens, [q,k,v] %d -> %d -> %d, SiLU, mean" % (L0.nQ, d3, dh, do),
                "ms": q_ms, "TFLOP/s": q_flops / (q_ms * 1e-3) / 1e12, "GB/s": q_bytes / (q_ms * 1e-3) / 1e9,
                "l2": "256 MB written between launches"}
-        del flush
 
     # ---- the paper's own schedule for pruning (Sec. 3.3): one Top-k at the final layer, its indices
     # applied to all 30 layers' caches in one launch (30 x 172.5 MB moved: far larger than L2)
@@ -494,46 +645,48 @@ def run_ours(args):
                "ms_with_attention_pass": e_f[0].elapsed_time(e_f[1])}
         del sQ, sK, sws, sO
 
+    # ---- the other measured configurations, inputs drawn on the device (same recipe): each is
+    # warmed up, timed with pafu_step alone in the timed region, split into kernels, clocks sampled
+    configs = None
+    if rank == 0 and world == 1 and args.all_configs and args.workload in ("wan1.3b_layer", "default") and n_layers == 1:
+        configs = {}
+        del layers
+        layers = None
+        torch.cuda.empty_cache()
+        # 30 independent layers (own cache, own head, own queries), retention budget 25 / 50 / 75 %
+        inputs = [wl.make_layer_device(wl.wan13b_layer(0.5), seed=0, layer=100 + l) for l in range(N_LAYERS_PER_DENOISE_STEP)]
+        for frac in (0.25, 0.5, 0.75):
+            wf = wl.wan13b_layer(frac)
+            ls = [Layer(wf, d, want_lse=False, want_slc=True) for d in inputs]
+            blk, _ = B.measure(wf, ls, N_LAYERS_PER_DENOISE_STEP, N_LAYERS_PER_DENOISE_STEP, steps=10, warmup=3, alone=False)
+            blk["workload"] = "30 independent Wan-1.3B-class layers, budget %d %% (%d of 28080 tokens kept)" % (round(100 * frac), wf.budget[0])
+            blk["ms_per_denoise_step"] = blk["ms_per_step"]
+            configs["wan1.3b_30layer_b%d" % round(100 * frac)] = blk
+            del ls
+        del inputs
+        torch.cuda.empty_cache()
+        for name, st, wu in (("long_horizon", 100, 5), ("batch4_14b", 20, 3)):
+            wc = wl.CONFIGS[name]()
+            ls = [Layer(wc, wl.make_layer_device(wc, seed=0, layer=l), want_lse=False, want_slc=True) for l in range(3)]
+            blk, _ = B.measure(wc, ls, 3, 1, steps=st, warmup=wu, alone=True)
+            configs[name] = blk
+            del ls
+            torch.cuda.empty_cache()
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    # a short timed region at full clock compares with the burst GEMM figure; a long one, or one
-    # whose sampled SM clock already sits at the power-capped level, with the sustained figure
-    capped = bool(clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and
-                  clocks["sm_mhz"] < 0.85 * clocks["sm_max_mhz"])
-    burst = total_ms < 1500.0 and not capped
-    peak_tf = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
-    attn_tf = work["attn_flops"] / (k_ms[3] * 1e-3) / 1e12
-    gbs = lambda b, ms: b / (ms * 1e-3) / 1e9
+    k = head["kernels_in_step"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "heads": w.n_heads, "d_head": w.d_head, "cache_tokens": list(w.T),
-                   "budget": list(w.budget), "n_sink": w.n_sink, "n_recent": w.n_recent,
-                   "chunk_tokens": list(w.Lq), "head_mlp": [w.d_model, w.d_hidden, w.d_out],
-                   "layers_per_step": n_layers,
-                   "l2": "inputs larger than L2: %d independent layer buffer sets (>= 300 MB each) used "
-                         "round-robin, no flush" % n_sets},
-        "roofline": {"kernel": "chunk attention", "bound": "tensor", "achieved": attn_tf, "peak": peak_tf,
-                     "unit": "TFLOP/s", "frac": attn_tf / peak_tf, "traffic": recorded_traffic(w),
-                     "peak_source": "%s, %s" % (peaks["source"], "burst" if burst else "sustained")},
-        "kernels": {
-            "score": {"ms": k_ms[0], "GB/s": gbs(work["score_bytes"], k_ms[0]),
-                      "TFLOP/s": work["score_flops"] / (k_ms[0] * 1e-3) / 1e12,
-                      "hbm_frac": gbs(work["score_bytes"], k_ms[0]) / peaks["hbm_gbs"]},
-            "select": {"ms": k_ms[1], "GB/s": gbs(work["select_bytes"], k_ms[1])},
-            "compact": {"ms": k_ms[2], "GB/s": gbs(work["compact_bytes"], k_ms[2]),
-                        "hbm_frac": gbs(work["compact_bytes"], k_ms[2]) / peaks["hbm_gbs"]},
-            "attn": {"ms": k_ms[3], "TFLOP/s": attn_tf, "tensor_frac": attn_tf / peak_tf},
-            "score+select+compact": {
-                "ms": float(k_ms[:3].sum()),
-                "GB/s": gbs(work["score_bytes"] + work["select_bytes"] + work["compact_bytes"], k_ms[:3].sum()),
-                "hbm_frac": gbs(work["score_bytes"] + work["select_bytes"] + work["compact_bytes"],
-                                k_ms[:3].sum()) / peaks["hbm_gbs"]},
-        },
+        "config": make_config(w, n_layers, n_sets),
+        "roofline": head["roofline"],
+        "kernels": k,
+        "kernels_alone": head.get("kernels_alone"),
         "score_qkv": qkv,
         "step_indexed": indexed,
         "cuda_graph": graph,
@@ -545,10 +698,11 @@ def run_ours(args):
         # cache once per chunk with the final layer's indices; every denoising step then only attends
         "paper_schedule": None if not (qkv and shared and args.shared_layers == N_LAYERS_PER_DENOISE_STEP) else {
             "prune_once_per_chunk_ms": qkv["ms"] + shared["ms"],
-            "attention_per_denoise_step_30_layers_ms": N_LAYERS_PER_DENOISE_STEP * float(k_ms[3]),
+            "attention_per_denoise_step_30_layers_ms": N_LAYERS_PER_DENOISE_STEP * k["attn"]["median"] * 1e-3,
             "note": "S-MLP on the chunk's [q,k,v] + one select + 30-layer shared-index compaction; "
                     "30 x (attention + merge) per denoising step"},
-        "peaks": peaks,
+        "configs": configs,
+        "peaks": dict(peaks, nominal=NOMINAL),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "api": "pafu_step_host (pinned host buffers)"},
@@ -576,6 +730,9 @@ def main():
                     help="layers pruned with one shared index list in the shared-index timing; 0 skips it")
     ap.add_argument("--graph", action=argparse.BooleanOptionalAction, default=True,
                     help="also time the steps replayed from a captured CUDA graph")
+    ap.add_argument("--all-configs", action=argparse.BooleanOptionalAction, default=True,
+                    help="after the headline, also measure the 30-layer budget sweep, the long-horizon cache "
+                         "and the batch-4 14B-class layer (single GPU, default workload only)")
     ap.add_argument("--sse-tokens", type=int, default=32760,
                     help="sequence length of the teacher-salience (Eq. 4/5) timing; 0 skips it")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

@@ -24,15 +24,16 @@ def bf16_to_bits(t: torch.Tensor) -> np.ndarray:
 class Layer:
     """All device buffers of one layer step for a workload."""
 
-    def __init__(self, w: Workload, data: Dict[str, np.ndarray], device="cuda", want_lse=True,
-                 want_slc=True):
+    def __init__(self, w: Workload, data: Dict[str, "np.ndarray | torch.Tensor"], device="cuda",
+                 want_lse=True, want_slc=True):
         self.w = w
         self.dev = torch.device(device)
         N, D = w.n_heads, w.d_head
         self.shape = B.Shape(N, D, w.cu("T"), w.cu("Lq"))
         self.policy = B.make_policy(w.n_sink, w.n_recent, list(w.budget), w.n_streams)
         self.cu_B = B.pafu_kept_counts(self.shape, self.policy)
-        up = lambda k: to_device_bf16(data[k], self.dev)
+        # numpy bf16 bit patterns are uploaded; tensors already on the device are used as they are
+        up = lambda k: data[k] if isinstance(data[k], torch.Tensor) else to_device_bf16(data[k], self.dev)
         self.K, self.V, self.Q, self.Kq, self.Vq = up("K"), up("V"), up("Q"), up("Kq"), up("Vq")
         self.w1, self.b1, self.w2, self.b2 = up("w1"), up("b1"), up("w2"), up("b2")
         self.head = B.Head(self.w1, self.b1, self.w2, self.b2, w.act, w.final)

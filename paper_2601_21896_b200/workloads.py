@@ -337,3 +337,58 @@ def queries_from_keys(w: Workload, d: Dict[str, np.ndarray], seed: int = 0) -> n
             else:
                 out[cuQ[s] + i] = d["Kq"][cuQ[s] + rng.integers(Lq)]
     return out
+
+
+def make_layer_device(w: Workload, seed: int = 0, layer: int = 0, device: str = "cuda"):
+    """The recipe of make_layer drawn on a CUDA device with torch's counter-based generator: the
+    same shapes, law and frame structure, a different random stream (the host version takes
+    seconds per layer at full size, which a 30-layer benchmark cannot afford).  Returns torch
+    bf16 tensors Q, K, V, Kq, Vq [tokens, n_heads, d_head] and w1, b1, w2, b2."""
+    import torch
+
+    N, D, dm = w.n_heads, w.d_head, w.d_model
+    g = torch.Generator(device=device)
+    g.manual_seed((int(seed) * 1000003 + int(w.wid) * 1009 + int(layer)) & 0x7FFFFFFF)
+    rn = lambda *shape: torch.randn(*shape, generator=g, device=device, dtype=torch.float32)
+
+    def tokens(n_tokens: int, first_frame: int, bases):
+        x = rn(n_tokens, dm)
+        if w.structure == "iid" or n_tokens == 0:
+            return x
+        tpf = w.tokens_per_frame
+        n_frames = (n_tokens + tpf - 1) // tpf
+        U = bases(first_frame + n_frames)[first_frame:]                    # [n_frames, rank, dm]
+        coef = rn(n_frames * tpf, w.rank).view(n_frames, tpf, w.rank)
+        shared = torch.bmm(coef, U).view(n_frames * tpf, dm)[:n_tokens]
+        return x + (w.shared_std / float(np.sqrt(w.rank))) * shared
+
+    out = {}
+    parts = {k: [] for k in ("Q", "K", "V", "Kq", "Vq")}
+    for s in range(w.n_streams):
+        first = (w.T[s] + w.tokens_per_frame - 1) // w.tokens_per_frame
+        n_total = first + (w.Lq[s] + w.tokens_per_frame - 1) // w.tokens_per_frame
+        cache = {}
+
+        def make_bases(tag):
+            def bases(n):
+                if tag not in cache:
+                    xi = rn(n_total, w.rank, dm)
+                    if w.structure == "lowrank_ar1":
+                        a, b = w.rho, float(np.sqrt(1.0 - w.rho * w.rho))
+                        for f in range(1, n_total):
+                            xi[f] = a * xi[f - 1] + b * xi[f]
+                    cache[tag] = xi
+                return cache[tag][:n]
+            return bases
+        bk, bv = make_bases("K"), make_bases("V")
+        parts["Q"].append(rn(w.Lq[s], dm))
+        parts["K"].append(tokens(w.T[s], 0, bk)); parts["V"].append(tokens(w.T[s], 0, bv))
+        parts["Kq"].append(tokens(w.Lq[s], first, bk)); parts["Vq"].append(tokens(w.Lq[s], first, bv))
+        del cache
+    for k, v in parts.items():
+        out[k] = torch.cat(v, dim=0).to(torch.bfloat16).view(-1, N, D).contiguous()
+    out["w1"] = (rn(w.d_hidden, dm) / float(np.sqrt(dm))).to(torch.bfloat16)
+    out["b1"] = (rn(w.d_hidden) / float(np.sqrt(dm))).to(torch.bfloat16)
+    out["w2"] = (rn(w.d_out, w.d_hidden) / float(np.sqrt(w.d_hidden))).to(torch.bfloat16)
+    out["b2"] = (rn(w.d_out) / float(np.sqrt(w.d_hidden))).to(torch.bfloat16)
+    return out
