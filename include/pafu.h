@@ -109,7 +109,10 @@ pafu_status pafu_kept_counts(const pafu_shape* shape, const pafu_policy* policy,
 /* Bytes of device scratch that pafu_score / pafu_select / pafu_chunk_attn / pafu_step need
  * for this geometry (`head` and `policy` may be NULL when the corresponding step is not
  * used).  Returns 0 on invalid arguments.  The workspace must be 256-byte aligned; its
- * first 256 bytes are a status header which the caller zeroes once after allocating. */
+ * first 256 bytes are a status header which the caller zeroes once after allocating.  The
+ * library keeps a time-out code, diagnostic counters and the work counters of pafu_step's row
+ * gather there (the latter return to zero at the end of every call); one workspace serves one
+ * call at a time - calls that may overlap on the GPU need a workspace each. */
 size_t pafu_workspace_bytes(const pafu_shape* shape, const pafu_policy* policy,
                             const pafu_head* head);
 
@@ -296,9 +299,12 @@ pafu_status pafu_step(const pafu_step_args* args, void* stream);
 pafu_status pafu_step_indexed(const pafu_step_args* args, void* stream);
 
 /* pafu_step with timestamps: identical launches, plus five caller-created CUDA events
- * (HOST array of 5 cudaEvent_t passed as void*) recorded on `stream` before the score step and
- * after the score, select, compact and attention steps.  Lets a caller attribute the step's
- * time to its kernels without changing what runs. */
+ * (HOST array of 5 cudaEvent_t passed as void*) recorded on `stream`: events 0 and 1 around the
+ * score step, events 2 and 3 around selection + row gather (two launches that overlap: the
+ * gather copies the always-kept rows while the selection runs, so no event can sit between
+ * them; event 2 follows event 1 at once), event 4 after the attention.  Lets a caller attribute
+ * the step's time to its kernels.  The events between the kernels do cost the overlap of each
+ * kernel's set-up with its predecessor's end, so the parts sum to slightly more than pafu_step. */
 pafu_status pafu_step_timed(const pafu_step_args* args, void* const* events, void* stream);
 
 /* Bytes of device memory pafu_step_host needs as its arena for this geometry. */

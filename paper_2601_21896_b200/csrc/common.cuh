@@ -29,6 +29,8 @@ constexpr int kStatusWordRescale = 10;     // output accumulator and row sum res
 // Test hook: while this word is non-zero the attention kernel's loader role issues no copies, so
 // every consumer's bounded wait runs out and the kernel unwinds with PAFU_ERR_TIMEOUT.
 constexpr int kStatusWordStallLoader = 32;
+// Work counters of the row gather inside a layer step (three words; back to zero when it ends).
+constexpr int kStatusWordGatherWork = 16;
 
 inline pafu_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? PAFU_OK : PAFU_ERR_CUDA; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -109,11 +111,12 @@ pafu_status launch_score(const pafu_head& head, const uint16_t* const* X, int n_
                          float* scores, void* ws, size_t ws_bytes, cudaStream_t stream);
 pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* idx,
                           cudaStream_t stream);
-// always_first: the rows that are kept whatever the scores say are copied before the kernel waits
-// for its predecessor (only valid when that predecessor is launch_select of the same step)
+// work != nullptr (three zeroed words of the workspace header): the rows that are kept whatever
+// the scores say are copied before the kernel waits for its predecessor (only valid when that
+// predecessor is launch_select of the same step)
 pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL,
                            const int32_t* idx, const StreamTable& st, int32_t d_model,
-                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream, bool always_first = false);
+                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream, int* work = nullptr);
 pafu_status launch_compact_layers(const uint16_t* const* K, const uint16_t* const* V, int32_t n_layers,
                                   const float* SL, const int32_t* idx, const StreamTable& st, int32_t d_model,
                                   uint16_t* const* Kc, uint16_t* const* Vc, float* SLc, cudaStream_t stream);

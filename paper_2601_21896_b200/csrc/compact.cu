@@ -44,23 +44,35 @@ __device__ __forceinline__ void copy_kv_row(const uint4* __restrict__ K, const u
 }
 
 // always_first = 0: wait for the preceding kernel, then copy every kept row through the index list.
-// always_first = 1 (inside a layer step, directly behind the selection kernel, which lets its
+// always_first = 1 (inside a layer step, directly behind the selection kernels, which let their
 // dependents start at once): the rows that are kept whatever the scores say - sink and recent
 // tokens, and all tokens of a stream that keeps everything - are copied first, while the
-// selection still runs on its one SM per stream; only then does the kernel wait for the indices
-// and copy the top-k rows.  K and V are not written by the step's earlier kernels, and the
-// outputs are not read by them, so the early part touches nothing the predecessor produces.
-// (SL is the score array in a step: all of its entries are copied after the wait.)
+// selection still runs on its few SMs; only then does the kernel wait for the indices and copy
+// the top-k rows.  K and V are not written by the step's earlier kernels, and the outputs are
+// not read by them, so the early part touches nothing the predecessor produces.  (SL is the
+// score array in a step: all of its entries are copied after the wait.)
+// In that mode rows are handed out through two counters in the workspace header (`work`: early
+// rows, late rows, finished blocks), four rows per claim: the blocks that only get an SM when
+// the selection's CTAs leave simply find less work left, instead of starting a fixed share late.
+// The last block to finish puts the counters back to zero.
+constexpr int kCompactClaim = 4;
+
+__device__ __forceinline__ int64_t claim_rows(int* counter, int lane) {
+    int v = 0;
+    if (lane == 0) v = atomicAdd(counter, kCompactClaim);
+    return __shfl_sync(0xffffffffu, v, 0);
+}
+
 __global__ void __launch_bounds__(kCompactWarpsPerBlock * 32)
 compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
                     const float* __restrict__ SL, const int32_t* __restrict__ idx,
                     const __grid_constant__ StreamTable st, int32_t chunks_per_row,
                     uint4* __restrict__ Kc, uint4* __restrict__ Vc, float* __restrict__ SLc,
-                    int64_t n_rows, int always_first) {
+                    int64_t n_rows, int* __restrict__ work) {
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = (int64_t)blockIdx.x * kCompactWarpsPerBlock + (threadIdx.x >> 5);
     const int64_t n_warps = (int64_t)gridDim.x * kCompactWarpsPerBlock;
-    if (!always_first) {
+    if (work == nullptr) {
         grid_dep_wait();
         for (int64_t r = warp0; r < n_rows; r += n_warps) {
             int s = 0;
@@ -75,20 +87,24 @@ compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
         const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
         n_always += B >= T ? T : st.n_sink[s] + st.n_recent[s];
     }
-    for (int64_t a = warp0; a < n_always; a += n_warps) {
-        int s = 0;
-        int64_t p = a;
-        for (;; ++s) {
+    // the next claim is always under way while the current rows are copied
+    for (int64_t base = claim_rows(work + 0, lane), next; base < n_always; base = next) {
+        next = claim_rows(work + 0, lane);
+        for (int64_t a = base; a < base + kCompactClaim && a < n_always; ++a) {
+            int s = 0;
+            int64_t p = a;
+            for (;; ++s) {
+                const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
+                const int64_t A = B >= T ? T : st.n_sink[s] + st.n_recent[s];
+                if (p < A) break;
+                p -= A;
+            }
             const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
-            const int64_t A = B >= T ? T : st.n_sink[s] + st.n_recent[s];
-            if (p < A) break;
-            p -= A;
+            const int64_t ns = B >= T ? T : st.n_sink[s], k = B >= T ? 0 : st.k[s], A = B >= T ? T : ns + st.n_recent[s];
+            // position p < ns is token p; position ns + k + i is token T - n_recent + i
+            const int64_t pos = p < ns ? p : p + k, tok = p < ns ? p : T - A + p;
+            copy_kv_row(K, V, nullptr, st.cu_T[s] + tok, st.cu_B[s] + pos, chunks_per_row, Kc, Vc, nullptr, lane);
         }
-        const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
-        const int64_t ns = B >= T ? T : st.n_sink[s], k = B >= T ? 0 : st.k[s], A = B >= T ? T : ns + st.n_recent[s];
-        // position p < ns is token p; position ns + k + i is token T - n_recent + i
-        const int64_t pos = p < ns ? p : p + k, tok = p < ns ? p : T - A + p;
-        copy_kv_row(K, V, nullptr, st.cu_T[s] + tok, st.cu_B[s] + pos, chunks_per_row, Kc, Vc, nullptr, lane);
     }
     // part 2: the selection's result
     grid_dep_wait();
@@ -102,12 +118,22 @@ compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
     }
     int64_t n_top = 0;
     for (int s = 0; s < st.n_streams; ++s) n_top += st.k[s];
-    for (int64_t q = warp0; q < n_top; q += n_warps) {
-        int s = 0;
-        int64_t p = q;
-        for (; p >= st.k[s]; ++s) p -= st.k[s];
-        const int64_t r = st.cu_B[s] + st.n_sink[s] + p;
-        copy_kv_row(K, V, SL, st.cu_T[s] + (int64_t)__ldg(idx + r), r, chunks_per_row, Kc, Vc, SLc, lane);
+    for (int64_t base = claim_rows(work + 1, lane), next; base < n_top; base = next) {
+        next = claim_rows(work + 1, lane);
+        for (int64_t q = base; q < base + kCompactClaim && q < n_top; ++q) {
+            int s = 0;
+            int64_t p = q;
+            for (; p >= st.k[s]; ++s) p -= st.k[s];
+            const int64_t r = st.cu_B[s] + st.n_sink[s] + p;
+            copy_kv_row(K, V, SL, st.cu_T[s] + (int64_t)__ldg(idx + r), r, chunks_per_row, Kc, Vc, SLc, lane);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(work + 2, 1) == (int)gridDim.x - 1) {      // every block is past its last claim
+            work[0] = 0; work[1] = 0; work[2] = 0;
+        }
     }
 }
 
@@ -176,26 +202,24 @@ pafu_status launch_compact_layers(const uint16_t* const* K, const uint16_t* cons
                                     lp, n_layers, SL, idx, st, d_model / 8, SLc, n_rows));
 }
 
+// `work`: three zeroed 32-bit words of device memory (the step's workspace header) - then the
+// always-kept rows are copied before the kernel waits for its predecessor, which must be
+// launch_select of the same step; nullptr: plain gather after the predecessor.
 pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL,
                            const int32_t* idx, const StreamTable& st, int32_t d_model,
-                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream, bool always_first) {
+                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream, int* work) {
     const int64_t n_rows = st.cu_B[st.n_streams];
     if (n_rows == 0) return PAFU_OK;
     const int32_t chunks = d_model / 8;
     int64_t blocks = (n_rows + kCompactWarpsPerBlock - 1) / kCompactWarpsPerBlock;
-    // A few resident waves, larger inputs loop.  With the early part every block must be resident
-    // from the start: a block that is waiting for the selection keeps its place on the SM, so a
-    // block behind it would reach its early rows only when the selection is over and would then
-    // finish its whole share late.  Three blocks fit on an SM, and the SMs that run the selection's
-    // CTAs (one per stream) take none.
-    int sms_free = device_sm_count() - st.n_streams;
-    if (sms_free < 1) sms_free = 1;
-    const int64_t max_blocks = always_first ? (int64_t)sms_free * 3 : 148 * 8 * 4;
+    // A few resident waves, larger inputs loop.  With the early part the grid is what the device
+    // holds at once (three blocks fit on an SM): a block must not queue behind blocks that are
+    // waiting for the selection.
+    const int64_t max_blocks = work != nullptr ? (int64_t)device_sm_count() * 3 : 148 * 8 * 4;
     if (blocks > max_blocks) blocks = max_blocks;
     return cuda_ok(launch_dependent(compact_rows_kernel, dim3((unsigned)blocks), dim3(kCompactWarpsPerBlock * 32), 0, stream, 1,
                                     reinterpret_cast<const uint4*>(K), reinterpret_cast<const uint4*>(V), SL, idx, st,
-                                    chunks, reinterpret_cast<uint4*>(Kc), reinterpret_cast<uint4*>(Vc), SLc, n_rows,
-                                    always_first ? 1 : 0));
+                                    chunks, reinterpret_cast<uint4*>(Kc), reinterpret_cast<uint4*>(Vc), SLc, n_rows, work));
 }
 
 }  // namespace pafu
