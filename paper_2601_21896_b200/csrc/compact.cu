@@ -52,16 +52,17 @@ __device__ __forceinline__ void copy_kv_row(const uint4* __restrict__ K, const u
 // not read by them, so the early part touches nothing the predecessor produces.  (SL is the
 // score array in a step: all of its entries are copied after the wait.)
 // In that mode rows are handed out through two counters in the workspace header (`work`: early
-// rows, late rows, finished blocks), four rows per claim: the blocks that only get an SM when
+// rows, late rows, finished blocks), one row per claim (the next claim under way during the copy): the blocks that only get an SM when
 // the selection's CTAs leave simply find less work left, instead of starting a fixed share late.
 // The last block to finish puts the counters back to zero.
-constexpr int kCompactClaim = 4;
+constexpr int kCompactClaim = 1;
 
-__device__ __forceinline__ int64_t claim_rows(int* counter, int lane) {
-    int v = 0;
-    if (lane == 0) v = atomicAdd(counter, kCompactClaim);
-    return __shfl_sync(0xffffffffu, v, 0);
+// A claim in two halves: lane 0 issues the add; its result is fetched (and shared with the warp)
+// only when the rows are needed, so the trip to L2 overlaps the copying in between.
+__device__ __forceinline__ int claim_issue(int* counter, int lane) {
+    return lane == 0 ? atomicAdd(counter, kCompactClaim) : 0;
 }
+__device__ __forceinline__ int64_t claim_get(int pending) { return __shfl_sync(0xffffffffu, pending, 0); }
 
 __global__ void __launch_bounds__(kCompactWarpsPerBlock * 32)
 compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
@@ -88,8 +89,9 @@ compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
         n_always += B >= T ? T : st.n_sink[s] + st.n_recent[s];
     }
     // the next claim is always under way while the current rows are copied
-    for (int64_t base = claim_rows(work + 0, lane), next; base < n_always; base = next) {
-        next = claim_rows(work + 0, lane);
+    int pending = claim_issue(work + 0, lane);
+    for (int64_t base = claim_get(pending); base < n_always; base = claim_get(pending)) {
+        pending = claim_issue(work + 0, lane);
         for (int64_t a = base; a < base + kCompactClaim && a < n_always; ++a) {
             int s = 0;
             int64_t p = a;
@@ -118,8 +120,9 @@ compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
     }
     int64_t n_top = 0;
     for (int s = 0; s < st.n_streams; ++s) n_top += st.k[s];
-    for (int64_t base = claim_rows(work + 1, lane), next; base < n_top; base = next) {
-        next = claim_rows(work + 1, lane);
+    pending = claim_issue(work + 1, lane);
+    for (int64_t base = claim_get(pending); base < n_top; base = claim_get(pending)) {
+        pending = claim_issue(work + 1, lane);
         for (int64_t q = base; q < base + kCompactClaim && q < n_top; ++q) {
             int s = 0;
             int64_t p = q;
