@@ -14,7 +14,8 @@
  *   compact  KV <- Select(KV; ids), SL <- Select(SL; ids) (Algorithm 2).
  *   attn     P = softmax(Q K^T / sqrt(D)) (Sec. 3.2), O = P V over the retained
  *            cache followed by the chunk's own tokens (Eq. 2 / Eq. 7).
- *   sse      teacher-side salience target of Eq. 4 and Eq. 5.
+ *   sse      teacher-side salience target of Eq. 4 and Eq. 5 (and the same in Algorithm 3's
+ *            order: mean over heads before the maximum over queries).
  *
  * All token tensors are bf16 bit patterns (uint16), token-major
  * [tokens, n_heads, d_head]; they are widened exactly to fp64 and every sum is
@@ -257,6 +258,53 @@ void pafu_oracle_sse(const uint16_t *Q, const uint16_t *K, int64_t L, int32_t N,
         if (comp) { comp[j] = low[j]; comp[L + j] = diag[j]; comp[2 * L + j] = up[j]; }
     }
     free(low); free(diag); free(up);
+}
+
+/* --------------------------------------------- sse in Algorithm 3's order of operations ---
+ * Algorithm 3 takes the mean over heads BEFORE the maximum over queries (Eq. 4 as printed takes
+ * the maximum per head first and then the mean):
+ *   a[i,j]  = (1/N) sum_n P[n,i,j]
+ *   low_j   = max_{i : j <  l(i)} a[i,j],  diag_j = max_{i : l(i) <= j < h(i)} a[i,j],
+ *   up_j    = max_{i : j >= h(i)} a[i,j]   (an empty index set gives 0), then Eq. 5 as above.
+ * One query row at a time: the row's softmax per head is added into a buffer of L means.
+ */
+void pafu_oracle_sse_meanfirst(const uint16_t *Q, const uint16_t *K, int64_t L, int32_t N, int32_t D,
+                               int64_t LB, double scale, double *s, double *comp) {
+    double *low = (double *)calloc((size_t)L, sizeof(double));
+    double *diag = (double *)calloc((size_t)L, sizeof(double));
+    double *up = (double *)calloc((size_t)L, sizeof(double));
+    double *a = (double *)malloc(sizeof(double) * (size_t)L);
+    double *p = (double *)malloc(sizeof(double) * (size_t)L);
+    const int64_t dm = (int64_t)N * D;
+    for (int64_t i = 0; i < L; ++i) {
+        for (int64_t j = 0; j < L; ++j) a[j] = 0.0;
+        for (int32_t n = 0; n < N; ++n) {
+            double m = -INFINITY;
+            for (int64_t j = 0; j < L; ++j) {
+                double acc = 0.0;
+                for (int32_t d = 0; d < D; ++d)
+                    acc += bf16_to_f64(Q[i * dm + n * D + d]) * bf16_to_f64(K[j * dm + n * D + d]);
+                p[j] = acc * scale;
+                if (p[j] > m) m = p[j];
+            }
+            double l = 0.0;
+            for (int64_t j = 0; j < L; ++j) { p[j] = exp(p[j] - m); l += p[j]; }
+            for (int64_t j = 0; j < L; ++j) a[j] += p[j] / l;
+        }
+        const int64_t lo = (i / LB) * LB, hi = lo + LB;
+        for (int64_t j = 0; j < L; ++j) {
+            const double v = a[j] / N;
+            double *dst = (j < lo) ? low : (j < hi) ? diag : up;
+            if (v > dst[j]) dst[j] = v;
+        }
+    }
+    for (int64_t j = 0; j < L; ++j) {
+        if (j < LB) s[j] = (diag[j] + low[j]) / 2.0;
+        else if (j < L - LB) s[j] = (up[j] + diag[j] + low[j]) / 3.0;
+        else s[j] = (diag[j] + up[j]) / 2.0;
+        if (comp) { comp[j] = low[j]; comp[L + j] = diag[j]; comp[2 * L + j] = up[j]; }
+    }
+    free(low); free(diag); free(up); free(a); free(p);
 }
 
 /* ------------------------------------------------------------- sse, sampled columns ---

@@ -61,6 +61,8 @@ def _load():
         lib.pafu_oracle_sse.argtypes = [_c_u16p, _c_u16p, ctypes.c_int64, ctypes.c_int32,
                                         ctypes.c_int32, ctypes.c_int64, ctypes.c_double, _c_f64p,
                                         _c_f64p]
+        lib.pafu_oracle_sse_meanfirst.restype = None
+        lib.pafu_oracle_sse_meanfirst.argtypes = lib.pafu_oracle_sse.argtypes
         lib.pafu_oracle_sse_gmax.restype = None
         lib.pafu_oracle_sse_gmax.argtypes = [_c_u16p, _c_u16p, ctypes.c_int64, ctypes.c_int32,
                                              ctypes.c_int32, ctypes.c_double, _c_f64p, _c_f64p]
@@ -171,6 +173,21 @@ def sse(Q: np.ndarray, K: np.ndarray, block_len: int, scale: Optional[float] = N
     comp = np.empty((3, L), dtype=np.float64)
     _load().pafu_oracle_sse(_p(Q, _c_u16p), _p(K, _c_u16p), L, N, D, block_len, float(scale),
                             _p(s, _c_f64p), _p(comp, _c_f64p))
+    return s, comp
+
+
+def sse_mean_first(Q: np.ndarray, K: np.ndarray, block_len: int, scale: Optional[float] = None
+                   ) -> Tuple[np.ndarray, np.ndarray]:
+    """The salience target in Algorithm 3's order (mean over heads, then the maximum over the
+    queries of each block class): s [L] and components [3, L] = low, diag, up."""
+    Q = _u16(Q); K = _u16(K)
+    L, N, D = Q.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(D)
+    s = np.empty(L, dtype=np.float64)
+    comp = np.empty((3, L), dtype=np.float64)
+    _load().pafu_oracle_sse_meanfirst(_p(Q, _c_u16p), _p(K, _c_u16p), L, N, D, block_len, float(scale),
+                                      _p(s, _c_f64p), _p(comp, _c_f64p))
     return s, comp
 
 

@@ -408,3 +408,41 @@ def test_sse_global_max_against_dense_torch():
     # it dominates each of the three block-wise components and equals their maximum for one head
     _, comp = oracle.sse(Q[:, :1], K[:, :1], 5)
     assert np.allclose(oracle.sse_global_max(Q[:, :1], K[:, :1]), comp.max(axis=0), atol=1e-14)
+
+
+def test_sse_mean_first_against_dense_torch_and_index_sets():
+    """Algorithm 3's order: the mean over heads comes before the maximum over queries.  Pinned to
+    dense torch softmax with the three query classes written as masks, to the explicit index sets
+    in Python loops, to the one-head case (where both orders are the same thing) and to the
+    inequality max_i mean_n P <= mean_n max_i P."""
+    rng = np.random.default_rng(33)
+    L, N, D, LB = 23, 3, 8, 6
+    Q = bf(rng.standard_normal((L, N, D)).astype(np.float32) * 2)
+    K = bf(rng.standard_normal((L, N, D)).astype(np.float32) * 2)
+    s, comp = oracle.sse_mean_first(Q, K, LB)
+    tq = torch.from_numpy(f32(Q)).double(); tk = torch.from_numpy(f32(K)).double()
+    A = torch.softmax(torch.einsum("qnd,knd->nqk", tq, tk) / math.sqrt(D), dim=-1).mean(dim=0).numpy()   # [L, L]
+    qi = np.arange(L)[:, None]; kj = np.arange(L)[None, :]
+    lo = (qi // LB) * LB; hi = lo + LB
+    low = np.where(kj < lo, A, 0).max(0); diag = np.where((kj >= lo) & (kj < hi), A, 0).max(0)
+    up = np.where(kj >= hi, A, 0).max(0)
+    assert np.allclose(comp, np.stack([low, diag, up]), atol=1e-13)
+    want = np.where(kj[0] < LB, (diag + low) / 2, np.where(kj[0] < L - LB, (up + diag + low) / 3, (diag + up) / 2))
+    assert np.allclose(s, want, atol=1e-13)
+    # explicit index sets
+    for j in range(L):
+        blk = lambda i: i // LB
+        sets = ([i for i in range(L) if blk(i) > blk(j)], [i for i in range(L) if blk(i) == blk(j)],
+                [i for i in range(L) if blk(i) < blk(j)])
+        for c, I in enumerate(sets):
+            assert abs(comp[c, j] - max((A[i, j] for i in I), default=0.0)) < 1e-13
+    # never above the per-head-maximum-first value of Eq. 4, and different from it for several heads
+    s4, comp4 = oracle.sse(Q, K, LB)
+    assert np.all(comp <= comp4 + 1e-15) and np.abs(comp - comp4).max() > 1e-3
+    # one head: the two orders coincide
+    s1, c1 = oracle.sse_mean_first(Q[:, :1], K[:, :1], LB)
+    s1b, c1b = oracle.sse(Q[:, :1], K[:, :1], LB)
+    assert np.allclose(c1, c1b, atol=1e-15) and np.allclose(s1, s1b, atol=1e-15)
+    # uniform attention (zero queries): every class that has queries gives 1 / L
+    _, cu = oracle.sse_mean_first(np.zeros_like(Q), K, LB)
+    assert np.allclose(cu[1], 1.0 / L, atol=1e-15)
