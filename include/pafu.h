@@ -350,6 +350,19 @@ pafu_status pafu_sse(const uint16_t* Q, const uint16_t* K, const float* LSE, int
                      int32_t n_heads, int32_t d_head, int64_t block_len, float scale,
                      float* s, float* comp, float* gmax, float* gavg, void* ws, size_t ws_bytes, void* stream);
 
+/* The salience target in Algorithm 3's order of operations.  Algorithm 3 averages the attention
+ * weights over the heads BEFORE it takes the maximum over a block class's queries, while Eq. 4
+ * takes each head's maximum first and then the mean (pafu_sse follows Eq. 4; for one head the two
+ * are the same).  With a[i,j] = mean over heads of P[n,i,j]:
+ *   low_j / diag_j / up_j = max of a[i,j] over the queries i of later / the same / earlier blocks
+ * and s_j by Eq. 5 as in pafu_sse.  Every value is <= the corresponding value of pafu_sse.
+ * Arguments as pafu_sse (without gmax and gavg); the workspace is the one of
+ * pafu_sse_workspace_bytes.  Needs one exponential per (query, key, head) and runs on mma.sync
+ * tiles: a comparison variant, several times slower than pafu_sse. */
+pafu_status pafu_sse_mean_first(const uint16_t* Q, const uint16_t* K, const float* LSE, int64_t L,
+                                int32_t n_heads, int32_t d_head, int64_t block_len, float scale,
+                                float* s, float* comp, void* ws, size_t ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -29,7 +29,7 @@ STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET
 EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
            "pafu_workspace_status", "pafu_workspace_counters", "pafu_score", "pafu_score_qkv", "pafu_select", "pafu_compact",
            "pafu_chunk_attn", "pafu_chunk_attn_indexed", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_indexed", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host",
-           "pafu_sse_workspace_bytes", "pafu_sse", "pafu_compact_layers"]
+           "pafu_sse_workspace_bytes", "pafu_sse", "pafu_sse_mean_first", "pafu_compact_layers"]
 
 
 class PafuError(RuntimeError):
@@ -121,6 +121,8 @@ def lib() -> ctypes.CDLL:
         L.pafu_sse_workspace_bytes.argtypes = [i64, i32, i32, i64]
         L.pafu_sse.restype = i32
         L.pafu_sse.argtypes = [vp, vp, vp, i64, i32, i32, i64, ctypes.c_float, vp, vp, vp, vp, vp, sz, vp]
+        L.pafu_sse_mean_first.restype = i32
+        L.pafu_sse_mean_first.argtypes = [vp, vp, vp, i64, i32, i32, i64, ctypes.c_float, vp, vp, vp, sz, vp]
         L.pafu_chunk_attn_noalloc.restype = i32
         L.pafu_chunk_attn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.POINTER(CShape),
                                               ctypes.c_float, vp, vp, vp]
@@ -314,6 +316,14 @@ def pafu_sse(Q, K, LSE, block_len: int, scale: float, s, comp, ws, gmax=None, ga
     L, N, D = Q.shape
     _check(lib().pafu_sse(_ptr(Q), _ptr(K), _ptr(LSE), L, N, D, block_len, float(scale), _ptr(s), _ptr(comp),
                           _ptr(gmax), _ptr(gavg), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pafu_sse")
+
+
+def pafu_sse_mean_first(Q, K, LSE, block_len: int, scale: float, s, comp, ws) -> None:
+    """The salience target with the mean over heads taken before the maximum over queries
+    (Algorithm 3's order); arguments as pafu_sse."""
+    L, N, D = Q.shape
+    _check(lib().pafu_sse_mean_first(_ptr(Q), _ptr(K), _ptr(LSE), L, N, D, block_len, float(scale), _ptr(s), _ptr(comp),
+                                     _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pafu_sse_mean_first")
 
 
 def pafu_step_indexed(args: CStepArgs) -> None:

@@ -546,6 +546,35 @@ def test_sse_matches_oracle(L, N, LB):
     assert torch.equal(s, s2)
 
 
+@pytest.mark.parametrize("L,N,LB", [
+    (700, 3, 200),      # four blocks, the last one half length; blocks and 64-token tiles do not line up
+    (1024, 2, 256),     # blocks that are whole tiles
+    (130, 1, 64),       # one head: Algorithm 3's order and Eq. 4's coincide
+])
+def test_sse_mean_first_matches_oracle(L, N, LB):
+    """Algorithm 3's order of operations (mean over heads, then the maximum over queries) against
+    its oracle; with one head also against pafu_sse itself."""
+    rng = np.random.default_rng(L * 7 + N)
+    D = 128
+    Q = wl.f32_to_bf16_bits((rng.standard_normal((L, N, D)) * 1.5).astype(np.float32))
+    K = wl.f32_to_bf16_bits((rng.standard_normal((L, N, D)) * 1.5).astype(np.float32))
+    want_s, want_c = oracle.sse_mean_first(Q, K, LB)
+    dQ, dK = to_device_bf16(Q), to_device_bf16(K)
+    ws = torch.zeros(pafu.pafu_sse_workspace_bytes(L, N, D, LB), dtype=torch.uint8, device="cuda")
+    s = torch.full((L,), float("nan"), device="cuda"); comp = torch.full((3, L), float("nan"), device="cuda")
+    pafu.pafu_sse_mean_first(dQ, dK, None, LB, 0.0, s, comp, ws)
+    assert pafu.pafu_workspace_status(ws) == 0
+    tol = dict(rtol=1e-3, atol=1e-7)
+    assert np.allclose(comp.cpu().numpy(), want_c, **tol), np.abs(comp.cpu().numpy() - want_c).max()
+    assert np.allclose(s.cpu().numpy(), want_s, **tol)
+    s4 = torch.full_like(s, float("nan")); comp4 = torch.full_like(comp, float("nan"))
+    pafu.pafu_sse(dQ, dK, None, LB, 0.0, s4, comp4, ws)
+    if N == 1:
+        assert np.allclose(comp.cpu().numpy(), comp4.cpu().numpy(), **tol)
+    else:
+        assert torch.all(comp <= comp4 * (1 + 1e-3) + 1e-7)       # max of the mean <= mean of the maxima
+
+
 def test_sse_full_size_sampled_columns():
     """The paper's training length (21 frames x 1560 tokens, blocks of 4680; Appendix A), one head:
     a seeded sample of key positions, block and tile boundaries included, against the oracle."""
