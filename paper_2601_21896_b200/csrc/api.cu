@@ -450,7 +450,7 @@ static pafu_status step_impl(const pafu_step_args* a, void* const* ev, void* str
         e = launch_select(a->scores, st, a->idx, cs);
         if (e != PAFU_OK) return e;
         e = launch_compact(a->K, a->V, a->SLc ? a->scores : nullptr, a->idx, st, (int32_t)dm, a->Kc, a->Vc, a->SLc, cs,
-                           static_cast<int*>(a->ws) + kStatusWordGatherWork);
+                           static_cast<int*>(a->ws) + kStatusWordGatherWork, select_cta_count(st));
         if (e != PAFU_OK) return e;
     } else {
         e = pafu_select(a->scores, &a->shape, a->policy, a->idx, a->ws, a->ws_bytes, stream);

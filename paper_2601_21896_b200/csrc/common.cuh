@@ -111,12 +111,14 @@ pafu_status launch_score(const pafu_head& head, const uint16_t* const* X, int n_
                          float* scores, void* ws, size_t ws_bytes, cudaStream_t stream);
 pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* idx,
                           cudaStream_t stream);
+int select_cta_count(const StreamTable& st);      // CTAs launch_select's kernels occupy for this geometry
 // work != nullptr (three zeroed words of the workspace header): the rows that are kept whatever
 // the scores say are copied before the kernel waits for its predecessor (only valid when that
 // predecessor is launch_select of the same step)
 pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL,
                            const int32_t* idx, const StreamTable& st, int32_t d_model,
-                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream, int* work = nullptr);
+                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream, int* work = nullptr,
+                           int select_ctas = 0);
 pafu_status launch_compact_layers(const uint16_t* const* K, const uint16_t* const* V, int32_t n_layers,
                                   const float* SL, const int32_t* idx, const StreamTable& st, int32_t d_model,
                                   uint16_t* const* Kc, uint16_t* const* Vc, float* SLc, cudaStream_t stream);

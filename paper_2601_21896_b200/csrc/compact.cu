@@ -51,10 +51,13 @@ __device__ __forceinline__ void copy_kv_row(const uint4* __restrict__ K, const u
 // the top-k rows.  K and V are not written by the step's earlier kernels, and the outputs are
 // not read by them, so the early part touches nothing the predecessor produces.  (SL is the
 // score array in a step: all of its entries are copied after the wait.)
-// In that mode rows are handed out through two counters in the workspace header (`work`: early
-// rows, late rows, finished blocks), one row per claim (the next claim under way during the copy): the blocks that only get an SM when
-// the selection's CTAs leave simply find less work left, instead of starting a fixed share late.
-// The last block to finish puts the counters back to zero.
+// When the selection occupies more than two SMs, rows are handed out through two counters in the
+// workspace header (`work`: early rows, late rows, finished blocks), one row per claim with the
+// next claim under way during the copy: the blocks that only get an SM when the selection's CTAs
+// leave simply find less work left, instead of starting a fixed share late (that tail cost 40 us
+// at the batch-4 size); the last block to finish puts the counters back to zero.  With a one- or
+// two-CTA selection the grid leaves those SMs out and every block takes a fixed share
+// (early_static; 5 us faster at the 28 080-token cache than claiming).
 constexpr int kCompactClaim = 1;
 
 // A claim in two halves: lane 0 issues the add; its result is fetched (and shared with the warp)
@@ -69,7 +72,7 @@ compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
                     const float* __restrict__ SL, const int32_t* __restrict__ idx,
                     const __grid_constant__ StreamTable st, int32_t chunks_per_row,
                     uint4* __restrict__ Kc, uint4* __restrict__ Vc, float* __restrict__ SLc,
-                    int64_t n_rows, int* __restrict__ work) {
+                    int64_t n_rows, int* __restrict__ work, int early_static) {
     const int lane = threadIdx.x & 31;
     const int64_t warp0 = (int64_t)blockIdx.x * kCompactWarpsPerBlock + (threadIdx.x >> 5);
     const int64_t n_warps = (int64_t)gridDim.x * kCompactWarpsPerBlock;
@@ -88,48 +91,59 @@ compact_rows_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
         const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
         n_always += B >= T ? T : st.n_sink[s] + st.n_recent[s];
     }
-    // the next claim is always under way while the current rows are copied
-    int pending = claim_issue(work + 0, lane);
-    for (int64_t base = claim_get(pending); base < n_always; base = claim_get(pending)) {
-        pending = claim_issue(work + 0, lane);
-        for (int64_t a = base; a < base + kCompactClaim && a < n_always; ++a) {
-            int s = 0;
-            int64_t p = a;
-            for (;; ++s) {
-                const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
-                const int64_t A = B >= T ? T : st.n_sink[s] + st.n_recent[s];
-                if (p < A) break;
-                p -= A;
-            }
+    auto copy_always = [&](int64_t a) {
+        int s = 0;
+        int64_t p = a;
+        for (;; ++s) {
             const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
-            const int64_t ns = B >= T ? T : st.n_sink[s], k = B >= T ? 0 : st.k[s], A = B >= T ? T : ns + st.n_recent[s];
-            // position p < ns is token p; position ns + k + i is token T - n_recent + i
-            const int64_t pos = p < ns ? p : p + k, tok = p < ns ? p : T - A + p;
-            copy_kv_row(K, V, nullptr, st.cu_T[s] + tok, st.cu_B[s] + pos, chunks_per_row, Kc, Vc, nullptr, lane);
+            const int64_t A = B >= T ? T : st.n_sink[s] + st.n_recent[s];
+            if (p < A) break;
+            p -= A;
         }
-    }
-    // part 2: the selection's result
-    grid_dep_wait();
-    if (SLc != nullptr) {
+        const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
+        const int64_t ns = B >= T ? T : st.n_sink[s], k = B >= T ? 0 : st.k[s], A = B >= T ? T : ns + st.n_recent[s];
+        // position p < ns is token p; position ns + k + i is token T - n_recent + i
+        const int64_t pos = p < ns ? p : p + k, tok = p < ns ? p : T - A + p;
+        copy_kv_row(K, V, nullptr, st.cu_T[s] + tok, st.cu_B[s] + pos, chunks_per_row, Kc, Vc, nullptr, lane);
+    };
+    auto copy_top = [&](int64_t q) {
+        int s = 0;
+        int64_t p = q;
+        for (; p >= st.k[s]; ++s) p -= st.k[s];
+        const int64_t r = st.cu_B[s] + st.n_sink[s] + p;
+        copy_kv_row(K, V, SL, st.cu_T[s] + (int64_t)__ldg(idx + r), r, chunks_per_row, Kc, Vc, SLc, lane);
+    };
+    int64_t n_top = 0;
+    for (int s = 0; s < st.n_streams; ++s) n_top += st.k[s];
+    auto fill_always_sl = [&]() {
+        if (SLc == nullptr) return;
         for (int64_t a = warp0 * 32 + lane; a < n_rows; a += n_warps * 32) {
             int s = 0;
             while (s + 1 < st.n_streams && a >= st.cu_B[s + 1]) ++s;
             const int64_t ns = st.n_sink[s], k = st.k[s], p = a - st.cu_B[s];
             if (k == 0 || p < ns || p >= ns + k) SLc[a] = __ldg(SL + st.cu_T[s] + __ldg(idx + a));
         }
+    };
+    if (early_static) {
+        // every block is resident from the start (the launcher sized the grid for it): fixed shares
+        for (int64_t a = warp0; a < n_always; a += n_warps) copy_always(a);
+        grid_dep_wait();
+        fill_always_sl();
+        for (int64_t q = warp0; q < n_top; q += n_warps) copy_top(q);
+        return;
     }
-    int64_t n_top = 0;
-    for (int s = 0; s < st.n_streams; ++s) n_top += st.k[s];
+    int pending = claim_issue(work + 0, lane);
+    for (int64_t base = claim_get(pending); base < n_always; base = claim_get(pending)) {
+        pending = claim_issue(work + 0, lane);
+        for (int64_t a = base; a < base + kCompactClaim && a < n_always; ++a) copy_always(a);
+    }
+    // part 2: the selection's result
+    grid_dep_wait();
+    fill_always_sl();
     pending = claim_issue(work + 1, lane);
     for (int64_t base = claim_get(pending); base < n_top; base = claim_get(pending)) {
         pending = claim_issue(work + 1, lane);
-        for (int64_t q = base; q < base + kCompactClaim && q < n_top; ++q) {
-            int s = 0;
-            int64_t p = q;
-            for (; p >= st.k[s]; ++s) p -= st.k[s];
-            const int64_t r = st.cu_B[s] + st.n_sink[s] + p;
-            copy_kv_row(K, V, SL, st.cu_T[s] + (int64_t)__ldg(idx + r), r, chunks_per_row, Kc, Vc, SLc, lane);
-        }
+        for (int64_t q = base; q < base + kCompactClaim && q < n_top; ++q) copy_top(q);
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -207,22 +221,27 @@ pafu_status launch_compact_layers(const uint16_t* const* K, const uint16_t* cons
 
 // `work`: three zeroed 32-bit words of device memory (the step's workspace header) - then the
 // always-kept rows are copied before the kernel waits for its predecessor, which must be
-// launch_select of the same step; nullptr: plain gather after the predecessor.
+// launch_select of the same step and runs on `select_ctas` CTAs; nullptr: plain gather after the
+// predecessor.
 pafu_status launch_compact(const uint16_t* K, const uint16_t* V, const float* SL,
                            const int32_t* idx, const StreamTable& st, int32_t d_model,
-                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream, int* work) {
+                           uint16_t* Kc, uint16_t* Vc, float* SLc, cudaStream_t stream, int* work, int select_ctas) {
     const int64_t n_rows = st.cu_B[st.n_streams];
     if (n_rows == 0) return PAFU_OK;
     const int32_t chunks = d_model / 8;
     int64_t blocks = (n_rows + kCompactWarpsPerBlock - 1) / kCompactWarpsPerBlock;
     // A few resident waves, larger inputs loop.  With the early part the grid is what the device
     // holds at once (three blocks fit on an SM): a block must not queue behind blocks that are
-    // waiting for the selection.
-    const int64_t max_blocks = work != nullptr ? (int64_t)device_sm_count() * 3 : 148 * 8 * 4;
+    // waiting for the selection.  Fixed shares: the selection's SMs are left out of the count.
+    const int early_static = work != nullptr && select_ctas <= 2;
+    int sms = device_sm_count() - (early_static ? select_ctas : 0);
+    if (sms < 1) sms = 1;
+    const int64_t max_blocks = work != nullptr ? (int64_t)sms * 3 : 148 * 8 * 4;
     if (blocks > max_blocks) blocks = max_blocks;
     return cuda_ok(launch_dependent(compact_rows_kernel, dim3((unsigned)blocks), dim3(kCompactWarpsPerBlock * 32), 0, stream, 1,
                                     reinterpret_cast<const uint4*>(K), reinterpret_cast<const uint4*>(V), SL, idx, st,
-                                    chunks, reinterpret_cast<uint4*>(Kc), reinterpret_cast<uint4*>(Vc), SLc, n_rows, work));
+                                    chunks, reinterpret_cast<uint4*>(Kc), reinterpret_cast<uint4*>(Vc), SLc, n_rows, work,
+                                    early_static));
 }
 
 }  // namespace pafu

@@ -120,23 +120,28 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
         fence_barrier_init();
     }
     if (warp == 8) { tmem_alloc(smem_u32(&tmem_base_sh), 512); tmem_relinquish(); }
-    grid_dep_wait();          // set-up above is local; everything below reads or writes global memory
-    // folded second layer and first-layer bias, fp32 in shared memory
-    for (int h = tid; h < p.d_hidden; h += kThreads) {
-        float m = 0.f;
-        for (int o = 0; o < p.d_out; ++o) m += bf16_bits(p.w2[(int64_t)o * p.d_hidden + h]);
-        w2m[h] = m / (float)p.d_out;
-        b1s[h] = p.b1 ? bf16_bits(p.b1[h]) : 0.f;
-    }
-    float b2m = 0.f;
-    if (p.b2) {
-        for (int o = 0; o < p.d_out; ++o) b2m += bf16_bits(p.b2[o]);
-        b2m /= (float)p.d_out;
-    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_base_sh;
+    grid_dep_wait();          // set-up above is local; everything below reads or writes global memory
+    // Folded second layer and first-layer bias, fp32 in shared memory: the read-out warps' business
+    // (they meet at a barrier of their own below), so the loader and the first MMAs do not wait
+    // for these global reads.
+    float b2m = 0.f;
+    if (warp < 8) {
+        for (int h = tid; h < p.d_hidden; h += 256) {
+            float m = 0.f;
+            for (int o = 0; o < p.d_out; ++o) m += bf16_bits(p.w2[(int64_t)o * p.d_hidden + h]);
+            w2m[h] = m / (float)p.d_out;
+            b1s[h] = p.b1 ? bf16_bits(p.b1[h]) : 0.f;
+        }
+        if (p.b2) {
+            for (int o = 0; o < p.d_out; ++o) b2m += bf16_bits(p.b2[o]);
+            b2m /= (float)p.d_out;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");    // unconditional and before any wait that can fail
+    }
 
     auto fail = [&](int code) {
         abort_flag = 1;

@@ -419,37 +419,53 @@ static_assert((kSelCapCta / kSelThreads) * (kSelThreads / 32) * 2 <= kSelHistBin
               "pair tables outgrow their buffers");
 }  // namespace
 
-pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* idx, cudaStream_t stream) {
-    if (st.n_streams == 0 || st.cu_B[st.n_streams] == 0) return PAFU_OK;
+namespace {
+struct SelLaunch {
     bool any_cluster = false, any_stream = false;
+    int nc = 1;
+    int64_t per_cta = 0;
+};
+SelLaunch plan_select(const StreamTable& st) {
+    SelLaunch pl;
     int64_t m_max = 0;
     for (int s = 0; s < st.n_streams; ++s) {
         const int64_t T = st.cu_T[s + 1] - st.cu_T[s], B = st.cu_B[s + 1] - st.cu_B[s];
         if (B == 0) continue;
         const int64_t M = B >= T ? 0 : T - st.n_sink[s] - st.n_recent[s];
-        if (M > kSelCapCluster) { any_stream = true; continue; }
-        any_cluster = true;
+        if (M > kSelCapCluster) { pl.any_stream = true; continue; }
+        pl.any_cluster = true;
         if (M > m_max) m_max = M;
     }
-    if (any_cluster) {
+    // CTAs per stream.  A barrier across CTAs and the trip through distributed shared memory cost
+    // more than a few rounds over the candidates: one CTA up to 24 rounds (24 576 candidates: the
+    // 28 080-token cache), then as many as keep a CTA's share near 16 rounds.
+    while (pl.nc < kSelCluster && m_max > (int64_t)pl.nc * (pl.nc == 1 ? 24576 : 16384)) pl.nc *= 2;
+    pl.per_cta = (m_max + pl.nc * kSelThreads - 1) / (pl.nc * kSelThreads) * kSelThreads;
+    return pl;
+}
+}  // namespace
+
+int select_cta_count(const StreamTable& st) {
+    const SelLaunch pl = plan_select(st);
+    return (pl.any_cluster ? st.n_streams * pl.nc : 0) + (pl.any_stream ? st.n_streams : 0);
+}
+
+pafu_status launch_select(const float* scores, const StreamTable& st, int32_t* idx, cudaStream_t stream) {
+    if (st.n_streams == 0 || st.cu_B[st.n_streams] == 0) return PAFU_OK;
+    const SelLaunch pl = plan_select(st);
+    if (pl.any_cluster) {
         static bool done[kMaxDevices] = {};
         if (!once_per_device(done, [] {
                 return cudaFuncSetAttribute(select_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelSmemMax) == cudaSuccess;
             }))
             return PAFU_ERR_CUDA;
-        // CTAs per stream.  A barrier across CTAs and the trip through distributed shared memory cost
-        // more than a few rounds over the candidates: one CTA up to 24 rounds (24 576 candidates: the
-        // 28 080-token cache), then as many as keep a CTA's share near 16 rounds.
-        int nc = 1;
-        while (nc < kSelCluster && m_max > (int64_t)nc * (nc == 1 ? 24576 : 16384)) nc *= 2;
-        const int64_t per_cta = (m_max + nc * kSelThreads - 1) / (nc * kSelThreads) * kSelThreads;
-        const int32_t keys_bytes = (int32_t)(per_cta * 4);
+        const int32_t keys_bytes = (int32_t)(pl.per_cta * 4);
         const size_t smem = (size_t)keys_bytes + kSelListCap * 4 + kSelHistBins * 4 * 2;
-        if (launch_dependent(select_cluster_kernel, dim3((unsigned)(st.n_streams * nc)), dim3(kSelThreads), smem, stream,
-                             (unsigned)nc, scores, st, keys_bytes, idx) != cudaSuccess)
+        if (launch_dependent(select_cluster_kernel, dim3((unsigned)(st.n_streams * pl.nc)), dim3(kSelThreads), smem, stream,
+                             (unsigned)pl.nc, scores, st, keys_bytes, idx) != cudaSuccess)
             return PAFU_ERR_CUDA;
     }
-    if (any_stream &&
+    if (pl.any_stream &&
         launch_dependent(select_stream_kernel, dim3((unsigned)st.n_streams), dim3(kSelThreads), 0, stream, 1, scores, st,
                          idx) != cudaSuccess)
         return PAFU_ERR_CUDA;
