@@ -47,6 +47,8 @@ struct Params {
     int d_in, d_hidden, d_out, act, final;
     int k_per_part;      // reduction slices (of kBK features) taken from each input matrix
     int split;           // 1: one (tile, chunk) per CTA, clusters of n_chunks CTAs
+    int tail_tiles;      // > 0: the last tail_tiles tiles are each split between the two CTAs of a cluster,
+    int tail_width;      //      tail_width hidden units per CTA (d_hidden / 2)
     const uint16_t* w2;
     const uint16_t* b1;
     const uint16_t* b2;
@@ -82,7 +84,7 @@ template <int ACT>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ CUtensorMap mX1,
                 const __grid_constant__ CUtensorMap mX2, const __grid_constant__ CUtensorMap mW,
-                const __grid_constant__ Params p) {
+                const __grid_constant__ CUtensorMap mWt, const __grid_constant__ Params p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sStage = smem_u32(smem);
@@ -106,11 +108,26 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
     const int64_t n_tiles = (p.n_tokens + kBM - 1) / kBM;
     const int n_chunks = (p.d_hidden + kNMax - 1) / kNMax;
     const int n_k = p.d_in / kBK;
-    // work of this CTA: tiles tile0, tile0 + tile_step, ... and chunks [ch0, ch1) of each
+    // Work of this CTA: tiles tile0, tile0 + tile_step, ... below n_main and chunks [ch0, ch1) of each;
+    // then, when the tiles do not fill the last round of CTAs, one "tail" unit: half of the hidden
+    // units of tile n_main + blockIdx / 2 (the two CTAs of a cluster share a tail tile, so the last
+    // round costs about two thirds of a full one instead of leaving half of the SMs idle).
     const int64_t tile0 = p.split ? blockIdx.x / n_chunks : blockIdx.x;
     const int64_t tile_step = p.split ? n_tiles : gridDim.x;
     const int ch0 = p.split ? (int)(blockIdx.x % n_chunks) : 0;
     const int ch1 = p.split ? ch0 + 1 : n_chunks;
+    const int64_t n_main = n_tiles - p.tail_tiles;
+    const bool has_tail = p.tail_tiles > 0 && (int)(blockIdx.x >> 1) < p.tail_tiles;
+    const int tail_half = (int)(blockIdx.x & 1);
+    const int64_t tail_tile = n_main + (blockIdx.x >> 1);
+    // the i-th tile-level unit of this CTA: false when there is none
+    struct Unit { int64_t tile; int c0, c1; bool tail; };
+    auto unit_at = [&](int64_t tile_next, bool tail_done, Unit& u) -> bool {
+        if (tile_next < n_main) { u.tile = tile_next; u.c0 = ch0; u.c1 = ch1; u.tail = false; return true; }
+        if (has_tail && !tail_done) { u.tile = tail_tile; u.c0 = 0; u.c1 = 1; u.tail = true; return true; }
+        return false;
+    };
+    const uint32_t tail_stage_bytes = kXBytes + (uint32_t)p.tail_width * kBK * 2;
 
     if (tid == 0) {
         for (int st = 0; st < kStages; ++st) { mbar_init(full(st), 1); mbar_init(empty(st), 1); }
@@ -153,20 +170,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
         if (elect_one()) {
             prefetch_tmap(&mX); prefetch_tmap(&mW);
             if (p.k_per_part < n_k) { prefetch_tmap(&mX1); prefetch_tmap(&mX2); }
+            prefetch_tmap(&mWt);
             uint32_t ring = 0;
             bool ok = true;
-            for (int64_t tile = tile0; tile < n_tiles && ok; tile += tile_step) {
-                for (int ch = ch0; ch < ch1 && ok; ++ch) {
+            Unit u;
+            int64_t tile_next = tile0;
+            for (bool tail_done = false; ok && unit_at(tile_next, tail_done, u); tile_next += tile_step, tail_done = u.tail) {
+                const int64_t tile = u.tile;
+                for (int ch = u.c0; ch < u.c1 && ok; ++ch) {
                     for (int k = 0; k < n_k; ++k, ++ring) {
                         const int st = ring % kStages;
                         if (abort_flag || !mbar_wait(empty(st), ((ring / kStages) & 1u) ^ 1u)) { fail(401); ok = false; break; }
                         const uint32_t dst = sStage + st * kStageBytes;
-                        mbar_arrive_expect_tx(full(st), kStageBytes);
+                        mbar_arrive_expect_tx(full(st), u.tail ? tail_stage_bytes : (uint32_t)kStageBytes);
                         // a token's features are the concatenation of its rows in up to three matrices
                         const int part = k / p.k_per_part;
                         const CUtensorMap* mx = part == 0 ? &mX : (part == 1 ? &mX1 : &mX2);
                         tma_load_2d(dst, mx, full(st), (k - part * p.k_per_part) * kBK, (int)(tile * kBM));
-                        tma_load_2d(dst + kXBytes, &mW, full(st), k * kBK, ch * kNMax);
+                        if (u.tail) tma_load_2d(dst + kXBytes, &mWt, full(st), k * kBK, tail_half * p.tail_width);
+                        else tma_load_2d(dst + kXBytes, &mW, full(st), k * kBK, ch * kNMax);
                     }
                 }
             }
@@ -181,10 +203,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
             const uint64_t desc0 = make_smem_desc_sw128(0, 16, 1024);
             uint32_t ring = 0, acc_it = 0;
             bool ok = true;
-            for (int64_t tile = tile0; tile < n_tiles && ok; tile += tile_step) {
-                for (int ch = ch0; ch < ch1 && ok; ++ch, ++acc_it) {
+            Unit u;
+            int64_t tile_next = tile0;
+            for (bool tail_done = false; ok && unit_at(tile_next, tail_done, u); tile_next += tile_step, tail_done = u.tail) {
+                for (int ch = u.c0; ch < u.c1 && ok; ++ch, ++acc_it) {
                     const int buf = acc_it & 1;
-                    const int nc = min(kNMax, p.d_hidden - ch * kNMax);
+                    const int nc = u.tail ? p.tail_width : min(kNMax, p.d_hidden - ch * kNMax);
                     const uint32_t idesc = make_idesc_bf16(kBM, nc, false, false);
                     if (abort_flag || !mbar_wait(acc_empty(buf), ((acc_it >> 1) & 1u) ^ 1u)) { fail(402); ok = false; break; }
                     tc_fence_after_sync();
@@ -211,11 +235,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
         const int row = quad * 32 + lane;
         uint32_t acc_it = 0, tile_it = 0;
         bool ok = true;
-        for (int64_t tile = tile0; tile < n_tiles && ok; tile += tile_step, ++tile_it) {
+        Unit u;
+        int64_t tile_next = tile0;
+        for (bool tail_done = false; ok && unit_at(tile_next, tail_done, u); tile_next += tile_step, tail_done = u.tail, ++tile_it) {
+            const int64_t tile = u.tile;
             float part = 0.f;
-            for (int ch = ch0; ch < ch1; ++ch, ++acc_it) {
+            for (int ch = u.c0; ch < u.c1; ++ch, ++acc_it) {
                 const int buf = acc_it & 1;
-                const int nc = min(kNMax, p.d_hidden - ch * kNMax);
+                const int nc = u.tail ? p.tail_width : min(kNMax, p.d_hidden - ch * kNMax);
+                const int h_base = u.tail ? tail_half * p.tail_width : ch * kNMax;    // first hidden unit of this accumulator
                 {
                     const bool w = mbar_wait(acc_full(buf), (acc_it >> 1) & 1u) && !abort_flag;
                     if (!__all_sync(0xffffffffu, w)) { fail(404); ok = false; break; }
@@ -226,7 +254,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
                     uint32_t r[16];
                     PAFU_TMEM_LD_X16(tmem + buf * kNMax + lane_base + g16 * 16, r);
                     tmem_wait_ld();
-                    const int h0 = ch * kNMax + g16 * 16;
+                    const int h0 = h_base + g16 * 16;
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
                         part = fmaf(w2m[h0 + i], act_fn<ACT>(__uint_as_float(r[i]) + b1s[h0 + i]), part);
@@ -236,7 +264,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
                 // the column-half-0 warps hand back a tile's last accumulator only after they have
                 // taken the other half's partial sums (below): the MMAs that reuse the accumulator, and
                 // with them the half-1 warps, can then never run two tiles ahead of a half-0 warp
-                if (lane == 0 && (half == 1 || ch + 1 < ch1)) mbar_arrive(acc_empty(buf));
+                if (lane == 0 && (half == 1 || ch + 1 < u.c1)) mbar_arrive(acc_empty(buf));
             }
             if (!ok) break;
             // combine the two column halves of each row
@@ -252,9 +280,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
                 __syncwarp();
                 if (lane == 0) mbar_arrive(acc_empty((acc_it - 1) & 1));
                 const int64_t t = tile * kBM + row;
-                if (p.split) {
-                    // this chunk's row sums go to the cluster's first CTA
-                    cooperative_groups::this_cluster().map_shared_rank(chunk_sum, 0)[ch0 * kBM + row] = part + other;
+                if (p.split || u.tail) {
+                    // this chunk's (this half's) row sums go to the cluster's first CTA
+                    cooperative_groups::this_cluster().map_shared_rank(chunk_sum, 0)[(u.tail ? tail_half : ch0) * kBM + row] = part + other;
                 } else if (t < p.n_tokens) {
                     float v = part + other + b2m;
                     if (p.final == PAFU_FINAL_SIGMOID) v = rcpf(1.0f + ex2f(-v * 1.4426950408889634f));
@@ -263,14 +291,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap mX, const __grid_constant__ 
             }
         }
     }
-    if (p.split) {
+    if (p.split || p.tail_tiles > 0) {
         // every thread of the cluster gets here (all loops above are bounded)
         cooperative_groups::this_cluster().sync();
-        if (ch0 == 0 && tid < kBM) {
-            const int64_t t = tile0 * kBM + tid;
+        const bool mine = p.split ? ch0 == 0 : (has_tail && tail_half == 0);
+        const int n_parts = p.split ? n_chunks : 2;
+        if (mine && tid < kBM) {
+            const int64_t t = (p.split ? tile0 : tail_tile) * kBM + tid;
             if (t < p.n_tokens) {
                 float v = chunk_sum[tid];
-                for (int c = 1; c < n_chunks; ++c) v += chunk_sum[c * kBM + tid];
+                for (int c = 1; c < n_parts; ++c) v += chunk_sum[c * kBM + tid];
                 v += b2m;
                 if (p.final == PAFU_FINAL_SIGMOID) v = rcpf(1.0f + ex2f(-v * 1.4426950408889634f));
                 p.scores[t] = v;
@@ -302,8 +332,21 @@ inline pafu_status launch(const pafu_head& head, const uint16_t* const* X, int n
     const int n_chunks = (head.d_hidden + kNMax - 1) / kNMax;
     // few tokens and a wide head: one CTA per (tile, chunk), clusters of n_chunks CTAs
     p.split = (n_chunks > 1 && n_tiles * n_chunks <= 2 * (int64_t)sm_count) ? 1 : 0;
-    const int grid = p.split ? (int)(n_tiles * n_chunks) : (int)(n_tiles < sm_count ? n_tiles : sm_count);
-    const unsigned cluster = p.split ? (unsigned)n_chunks : 1u;
+    // tiles that fill at most half of the last round of CTAs (220 tiles on 148 SMs leave 72): each
+    // is shared by the two CTAs of a cluster, half of the hidden units each
+    p.tail_tiles = 0; p.tail_width = 0;
+    const int64_t rest = n_tiles % sm_count;
+    if (!p.split && n_chunks == 1 && head.d_hidden % 32 == 0 && sm_count % 2 == 0 && rest > 0 && 2 * rest <= sm_count) {
+        p.tail_tiles = (int)rest;
+        p.tail_width = head.d_hidden / 2;
+    }
+    CUtensorMap mWt = mW;
+    if (p.tail_tiles > 0 &&
+        !TmapEncoder::matrix(&mWt, head.w1, (uint64_t)head.d_hidden, (uint64_t)head.d_in, (uint64_t)head.d_in, (uint32_t)p.tail_width))
+        return PAFU_ERR_CUDA;
+    int grid = p.split ? (int)(n_tiles * n_chunks) : (int)(n_tiles < sm_count ? n_tiles : sm_count);
+    if (p.tail_tiles > 0 && n_tiles < sm_count) grid = 2 * p.tail_tiles;      // no full round at all
+    const unsigned cluster = p.split ? (unsigned)n_chunks : (p.tail_tiles > 0 ? 2u : 1u);
     static bool attr_set[kMaxDevices] = {};
     if (!once_per_device(attr_set, [] {
             return cudaFuncSetAttribute(score_tc_kernel<PAFU_ACT_GELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess &&
@@ -311,8 +354,8 @@ inline pafu_status launch(const pafu_head& head, const uint16_t* const* X, int n
         }))
         return PAFU_ERR_CUDA;
     return cuda_ok(head.act == PAFU_ACT_GELU
-                       ? launch_dependent(score_tc_kernel<PAFU_ACT_GELU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, cluster, mX[0], mX[1], mX[2], mW, p)
-                       : launch_dependent(score_tc_kernel<PAFU_ACT_SILU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, cluster, mX[0], mX[1], mX[2], mW, p));
+                       ? launch_dependent(score_tc_kernel<PAFU_ACT_GELU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, cluster, mX[0], mX[1], mX[2], mW, mWt, p)
+                       : launch_dependent(score_tc_kernel<PAFU_ACT_SILU>, dim3(grid), dim3(kThreads), kSmemBytes, stream, cluster, mX[0], mX[1], mX[2], mW, mWt, p));
 }
 
 }  // namespace score_tc
