@@ -138,6 +138,40 @@ def test_newer_entry_points_reject_bad_arguments_on_host(L):
     assert sse(1000, 2, 128, 256, 0.0, fake, fake, need - 1) == 4
 
 
+def test_overlap_and_host_step_checks_run_before_anything_is_enqueued(L):
+    """Outputs that overlap inputs are rejected by range, not only by equal pointers; and the
+    host-buffer step validates the whole head before its first copy (every call below returns an
+    argument error with fake pointers that must never be touched)."""
+    fake = 0x7f0000000000
+    sh = pafu.Shape(2, 128, [0, 512], [0, 64])                 # 512 cache rows of 512 bytes, 128 kept
+    pol = pafu.make_policy(4, 64, 128, 1)
+    K, V = fake, fake + (1 << 20)
+    inside_K = fake + 512 * 512 - 1024                          # starts inside K's last rows
+    ok_Kc, ok_Vc = fake + (2 << 20), fake + (3 << 20)
+    cp = lambda Kc, Vc, SL=None, SLc=None: L.pafu_compact(K, V, SL, fake + (4 << 20), ctypes.byref(sh.c), pol, Kc, Vc, SLc, None)
+    assert cp(inside_K, ok_Vc) == 1                             # Kc overlaps K
+    assert cp(ok_Kc, V + 4096) == 1                             # Vc overlaps V
+    assert cp(ok_Kc, ok_Kc + 1024) == 1                         # the two outputs overlap each other
+    assert cp(ok_Kc, ok_Vc, fake + (5 << 20), fake + (5 << 20) + 256) == 1    # SLc inside SL
+    # host-buffer step: bad head sizes / enums / scale are caught before any copy
+    head = lambda d_in, d_hid, act: B.CHead(d_in, d_hid, 1, act, 0, fake, None, fake, None)
+    pol1 = ctypes.cast(pol, ctypes.POINTER(B.CPolicy))
+    def args(h, scale=0.0):
+        a = B.CStepArgs(sh.c, ctypes.pointer(h), pol1, fake, fake, fake, fake, fake, scale, fake, fake, None, None, None,
+                        fake, None, None, 0)
+        a._keep = h
+        return a
+    arena = 0x7f1000000000
+    big = 1 << 40
+    assert L.pafu_step_host(ctypes.byref(args(head(256, 17, 0))), arena, big, None) == 3     # d_hidden % 16
+    assert L.pafu_step_host(ctypes.byref(args(head(256, 32, 9))), arena, big, None) == 1     # activation enum
+    assert L.pafu_step_host(ctypes.byref(args(head(192, 32, 0))), arena, big, None) == 1     # d_in != heads * d_head
+    assert L.pafu_step_host(ctypes.byref(args(head(256, 32, 0), -1.0)), arena, big, None) == 1
+    assert L.pafu_step_host(ctypes.byref(args(head(256, 32, 0))), arena + 8, big, None) == 5  # arena alignment
+    assert L.pafu_step_host(ctypes.byref(args(head(256, 32, 0))), arena, 1024, None) == 4     # arena too small
+    assert L.pafu_workspace_counters(None, None, None) == 1
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
