@@ -321,6 +321,18 @@ size_t pafu_step_host_arena_bytes(const pafu_shape* shape, const pafu_policy* po
 pafu_status pafu_step_host(const pafu_step_args* args, void* arena, size_t arena_bytes,
                            void* stream);
 
+/* pafu_step_host without the final synchronisation, for callers that keep several steps in flight
+ * (two streams with an arena each: the copies of one step then overlap the kernels of the other
+ * and the host link, not the sum of link and kernels, sets the pace).  Everything is enqueued on
+ * `stream` and the call returns; the host outputs, and *timeout_word, are valid once the caller
+ * has synchronised `stream`.
+ *   timeout_word   HOST int32 (pinned memory for a truly asynchronous copy), out: 0, or the code of
+ *                  a bounded device wait that ran out (treat non-zero as PAFU_ERR_TIMEOUT)
+ * The argument structs, the prefix arrays and the host buffers must stay valid until then, and the
+ * arena must not be used by another call in the meantime. */
+pafu_status pafu_step_host_async(const pafu_step_args* args, void* arena, size_t arena_bytes,
+                                 void* stream, int32_t* timeout_word);
+
 /* Teacher-side salience target - Spatialtemporal-balanced Salience Estimation (Sec. 3.2, Eq. 4
  * and Eq. 5; Algorithm 3).  With P = softmax(scale * Q K^T) per head over the whole sequence of L
  * tokens (bidirectional) and blocks of block_len tokens, key j gets

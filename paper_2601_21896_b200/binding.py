@@ -28,7 +28,7 @@ STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET
 
 EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
            "pafu_workspace_status", "pafu_workspace_counters", "pafu_score", "pafu_score_qkv", "pafu_select", "pafu_compact",
-           "pafu_chunk_attn", "pafu_chunk_attn_indexed", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_indexed", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host",
+           "pafu_chunk_attn", "pafu_chunk_attn_indexed", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_indexed", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host", "pafu_step_host_async",
            "pafu_sse_workspace_bytes", "pafu_sse", "pafu_sse_mean_first", "pafu_compact_layers"]
 
 
@@ -135,6 +135,8 @@ def lib() -> ctypes.CDLL:
                                                  ctypes.POINTER(CHead)]
         L.pafu_step_host.restype = i32
         L.pafu_step_host.argtypes = [ctypes.POINTER(CStepArgs), vp, sz, vp]
+        L.pafu_step_host_async.restype = i32
+        L.pafu_step_host_async.argtypes = [ctypes.POINTER(CStepArgs), vp, sz, vp, vp]
         _lib = L
     return _lib
 
@@ -350,3 +352,11 @@ def pafu_step_host_arena_bytes(shape: Shape, policy, head: Head) -> int:
 def pafu_step_host(args: CStepArgs, arena: torch.Tensor) -> None:
     _check(lib().pafu_step_host(ctypes.byref(args), _ptr(arena),
                                 arena.numel() * arena.element_size(), _stream()), "pafu_step_host")
+
+
+def pafu_step_host_async(args: CStepArgs, arena: torch.Tensor, timeout_word: torch.Tensor, stream=None) -> None:
+    """pafu_step_host without the final synchronisation; timeout_word is a pinned int32 tensor of
+    one element, valid (like the host outputs) after the stream has been synchronised."""
+    st = _stream() if stream is None else stream.cuda_stream
+    _check(lib().pafu_step_host_async(ctypes.byref(args), _ptr(arena), arena.numel() * arena.element_size(), st,
+                                      _ptr(timeout_word)), "pafu_step_host_async")

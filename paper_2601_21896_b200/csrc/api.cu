@@ -511,7 +511,23 @@ size_t pafu_step_host_arena_bytes(const pafu_shape* shape, const pafu_policy* po
     return plan_host(shape, cu_B, head, ws).total;
 }
 
+static pafu_status step_host_impl(const pafu_step_args* a, void* arena, size_t arena_bytes, void* stream, int32_t* timeout_word);
+
 pafu_status pafu_step_host(const pafu_step_args* a, void* arena, size_t arena_bytes, void* stream) {
+    int32_t word = 0;
+    pafu_status e = step_host_impl(a, arena, arena_bytes, stream, &word);
+    if (e != PAFU_OK) return e;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return PAFU_ERR_CUDA;
+    return word == 0 ? PAFU_OK : PAFU_ERR_TIMEOUT;
+}
+
+pafu_status pafu_step_host_async(const pafu_step_args* a, void* arena, size_t arena_bytes, void* stream,
+                                 int32_t* timeout_word) {
+    if (timeout_word == nullptr) return PAFU_ERR_INVALID_ARG;
+    return step_host_impl(a, arena, arena_bytes, stream, timeout_word);
+}
+
+static pafu_status step_host_impl(const pafu_step_args* a, void* arena, size_t arena_bytes, void* stream, int32_t* timeout_word) {
     if (a == nullptr || arena == nullptr || a->head == nullptr) return PAFU_ERR_INVALID_ARG;
     pafu_status e = shape_ok(&a->shape, true, true);
     if (e != PAFU_OK) return e;
@@ -581,13 +597,10 @@ pafu_status pafu_step_host(const pafu_step_args* a, void* arena, size_t arena_by
     d.ws_bytes = p.ws_bytes;
     e = pafu_step(&d, stream);
     if (e != PAFU_OK) return e;
-    int32_t word = 0;
     ok = d2h(a->scores, p.scores, nT * 4) && d2h(a->idx, p.idx, nB * 4) && d2h(a->O, p.O, nQ * dm * 2) &&
          d2h(a->Kc, p.Kc, nB * dm * 2) && d2h(a->Vc, p.Vc, nB * dm * 2) && d2h(a->SLc, p.SLc, nB * 4) &&
-         d2h(a->LSE, p.LSE, nQ * a->shape.n_heads * 4) && d2h(&word, p.ws, 4);
-    if (!ok) return PAFU_ERR_CUDA;
-    if (cudaStreamSynchronize(cs) != cudaSuccess) return PAFU_ERR_CUDA;
-    return word == 0 ? PAFU_OK : PAFU_ERR_TIMEOUT;
+         d2h(a->LSE, p.LSE, nQ * a->shape.n_heads * 4) && d2h(timeout_word, p.ws, 4);
+    return ok ? PAFU_OK : PAFU_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -647,6 +647,40 @@ def test_step_host_matches_device_step():
     assert torch.equal(O, A.O.view(torch.int16).cpu())
 
 
+def test_step_host_async_two_steps_in_flight():
+    """Two host-buffer steps on two streams with an arena each (the copies of one overlap the
+    kernels of the other): after the streams are synchronised both give what the blocking call gives."""
+    w = wl.small_ragged(2, 128)
+    datas = [wl.make_layer(w, seed=s) for s in (0, 1)]
+    want = []
+    for d in datas:
+        A = Layer(w, d)
+        A.step(); A.check_status()
+        want.append((A.scores[: A.nT].cpu(), A.idx[: A.nB].cpu(), A.O.view(torch.int16).cpu()))
+    shape, policy, nT, nB, nQ = A.shape, A.policy, A.nT, A.nB, A.nQ
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    keep, outs = [], []
+    torch.cuda.synchronize()
+    for d, st in zip(datas, streams):
+        host = {k: torch.from_numpy(v.view(np.int16)).pin_memory() for k, v in d.items()}
+        scores = torch.empty(nT, dtype=torch.float32).pin_memory()
+        idx = torch.empty(nB, dtype=torch.int32).pin_memory()
+        O = torch.empty((nQ, w.n_heads, w.d_head), dtype=torch.int16).pin_memory()
+        word = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+        head = pafu.Head(host["w1"], host["b1"], host["w2"], host["b2"], w.act, w.final)
+        arena = torch.empty(pafu.pafu_step_host_arena_bytes(shape, policy, head), dtype=torch.uint8, device="cuda")
+        args = pafu.step_args(shape, head, policy, host["K"], host["V"], host["Q"], host["Kq"], host["Vq"],
+                              0.0, scores, idx, None, None, None, O, None, None)
+        pafu.pafu_step_host_async(args, arena, word, stream=st)
+        keep.append((host, head, arena, args))
+        outs.append((scores, idx, O, word))
+    for st in streams:
+        st.synchronize()
+    for (scores, idx, O, word), (ws, wi, wo) in zip(outs, want):
+        assert int(word[0]) == 0
+        assert torch.equal(scores, ws) and torch.equal(idx, wi) and torch.equal(O, wo)
+
+
 # ---------------------------------------------------------------------- full-size configs
 def _full_size_check(w, n_rows=256, seed=0, score_rows=None, peaked=False):
     d = wl.make_layer(w, seed=seed)
