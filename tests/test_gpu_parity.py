@@ -22,7 +22,7 @@ REL_FRO = 5e-3
 
 
 def close(got, want, what="", scaled=False):
-    """The benchmark spec's bounds (max-abs 2e-2, mean-abs 2e-3) plus the relative bound above.  `scaled`:
+    """The stated floating-point bounds (max-abs 2e-2, mean-abs 2e-3) plus the relative bound above.  `scaled`:
     the inputs were built to give outputs of magnitude up to ~4.5 (attention that picks single
     value rows); bf16 rounding of an output o alone is up to 2^-8 |o| = 1.8e-2 there, and the bf16
     probabilities add up to 2^-8 max|v|, so the absolute bounds grow with max|want|."""
