@@ -138,6 +138,33 @@ def compact(x: np.ndarray, idx: np.ndarray) -> np.ndarray:
     return out
 
 
+def cache_update(K, V, SL: np.ndarray, newK, newV, s_new: np.ndarray, capacity: int, n_sink: int):
+    """One chunk of the rolling-cache update of Algorithm 2, for every layer at once.
+
+    ``K``, ``V``: lists (one entry per layer) of arrays ``[T, ...]``; ``SL``: the salience list
+    ``[T]`` carried with the cache; ``newK``, ``newV``: the chunk's rows per layer ``[C, ...]``;
+    ``s_new``: the chunk's salience scores ``[C]``.  When the chunk no longer fits
+    (``T + C > capacity``) the cache is first pruned to ``capacity - C`` tokens: the sink prefix
+    and the highest entries of ``SL`` (ties to the lower index), ONE index list applied to
+    every layer's K and V and to ``SL`` itself; then the chunk and its scores are appended.
+    Returns ``(K, V, SL, ids)`` with ``ids`` the index list of the pruning, or None."""
+    SL = np.ascontiguousarray(SL, dtype=np.float32)
+    s_new = np.ascontiguousarray(s_new, dtype=np.float32)
+    T, C = SL.shape[0], s_new.shape[0]
+    if C > capacity:
+        raise ValueError("chunk longer than the cache")
+    ids = None
+    if T + C > capacity:
+        ids = select(SL, n_sink, 0, capacity - C)
+        K = [compact(k, ids) for k in K]
+        V = [compact(v, ids) for v in V]
+        SL = compact(SL, ids)
+    K = [np.concatenate([k, np.ascontiguousarray(n)]) for k, n in zip(K, newK)]
+    V = [np.concatenate([v, np.ascontiguousarray(n)]) for v, n in zip(V, newV)]
+    SL = np.concatenate([SL, s_new])
+    return K, V, SL, ids
+
+
 def attention(Q: np.ndarray, Kc: np.ndarray, Vc: np.ndarray, Kq: Optional[np.ndarray],
               Vq: Optional[np.ndarray], scale: Optional[float] = None,
               rows: Optional[Sequence[int]] = None) -> Tuple[np.ndarray, np.ndarray]:

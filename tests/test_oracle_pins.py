@@ -446,3 +446,46 @@ def test_sse_mean_first_against_dense_torch_and_index_sets():
     # uniform attention (zero queries): every class that has queries gives 1 / L
     _, cu = oracle.sse_mean_first(np.zeros_like(Q), K, LB)
     assert np.allclose(cu[1], 1.0 / L, atol=1e-15)
+
+
+def test_cache_update_is_algorithm2_by_brute_force():
+    """Algorithm 2's cache update against a brute-force statement of it: while the chunk fits
+    nothing moves; otherwise the survivors are the sink prefix plus the best of the rest by
+    (score descending, index ascending), in their old order, the same rows in every layer."""
+    rng = np.random.default_rng(5)
+    cap, C, n_sink, n_layers = 40, 12, 5, 3
+    K = [np.zeros((0, 4), np.uint16) for _ in range(n_layers)]; V = [k.copy() for k in K]
+    SL = np.zeros(0, np.float32)
+    tags = np.zeros(0, np.int64)                         # global token number of every cached row
+    next_tag, pruned = 0, 0
+    for c in range(9):
+        newK = [rng.integers(0, 65536, (C, 4)).astype(np.uint16) for _ in range(n_layers)]
+        newV = [rng.integers(0, 65536, (C, 4)).astype(np.uint16) for _ in range(n_layers)]
+        for l in range(n_layers):
+            newK[l][:, 0] = np.arange(next_tag, next_tag + C) & 0xffff     # row identity travels with the row
+        s_new = rng.integers(0, 6, C).astype(np.float32)                   # many ties
+        T = SL.shape[0]
+        K2, V2, SL2, ids = oracle.cache_update(K, V, SL, newK, newV, s_new, cap, n_sink)
+        if T + C <= cap:
+            assert ids is None
+            keep = np.arange(T)
+        else:
+            pruned += 1
+            k = cap - C
+            rest = sorted(range(n_sink, T), key=lambda i: (-SL[i], i))[: k - n_sink]
+            keep = np.array(sorted(list(range(n_sink)) + rest))
+            assert np.array_equal(ids, keep) and len(keep) == k
+        assert SL2.shape[0] == len(keep) + C <= cap
+        assert np.array_equal(SL2, np.concatenate([SL[keep], s_new]))
+        for l in range(n_layers):
+            assert np.array_equal(K2[l], np.concatenate([K[l][keep], newK[l]]))
+            assert np.array_equal(V2[l], np.concatenate([V[l][keep], newV[l]]))
+        tags = np.concatenate([tags[keep], np.arange(next_tag, next_tag + C)])
+        assert np.array_equal(K2[0][:, 0], tags & 0xffff)
+        assert np.array_equal(tags[:n_sink], np.arange(n_sink))            # the sink prefix never leaves
+        assert np.all(np.diff(tags) > 0)                                   # temporal order is kept
+        K, V, SL, next_tag = K2, V2, SL2, next_tag + C
+    assert pruned >= 5
+    with pytest.raises(ValueError):
+        oracle.cache_update(K, V, SL, [np.zeros((cap + 1, 4), np.uint16)] * n_layers,
+                            [np.zeros((cap + 1, 4), np.uint16)] * n_layers, np.zeros(cap + 1, np.float32), cap, n_sink)
