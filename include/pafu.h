@@ -52,7 +52,7 @@ enum {
     PAFU_ERR_MISALIGNED = 5,         /* a device pointer is not 16-byte aligned */
     PAFU_ERR_CUDA = 6,               /* a CUDA runtime/driver call failed (launch error, no device) */
     PAFU_ERR_TIMEOUT = 7,            /* a bounded device-side wait ran out (pafu_workspace_status) */
-    PAFU_ERR_TOO_LARGE = 8           /* problem exceeds the built-in scratch of pafu_chunk_attn_noalloc */
+    PAFU_ERR_TOO_LARGE = 8           /* exceeds pafu_chunk_attn_noalloc's built-in scratch, or a pafu_cache's capacity */
 };
 
 /* Activation between the two linear layers of the salience head. */
@@ -332,6 +332,47 @@ pafu_status pafu_step_host(const pafu_step_args* args, void* arena, size_t arena
  * arena must not be used by another call in the meantime. */
 pafu_status pafu_step_host_async(const pafu_step_args* args, void* arena, size_t arena_bytes,
                                  void* stream, int32_t* timeout_word);
+
+/* The rolling KV cache of Algorithm 2 for one stream and all layers, and its update once a chunk
+ * has been generated (Sec. 3.3: the salience head sits in the final layer and its Top-k prunes
+ * every layer's cache; Algorithm 2: "if |KV| = L: ids <- Top-k(SL); KV <- Select(KV; ids);
+ * SL <- Select(SL; ids)", then KV.append(kv), SL.append(s)).
+ * The cache lives in two sets of buffers; a pruning gathers from the current set into the other
+ * and makes that one current (rows are never moved inside a buffer).  All counters are host-side. */
+typedef struct pafu_cache {
+    int32_t n_layers;        /* <= PAFU_MAX_LAYERS */
+    int32_t n_heads, d_head; /* n_heads * d_head % 8 == 0 */
+    int32_t cur;             /* in/out: which buffer set (0 or 1) holds the cache */
+    int64_t capacity;        /* L: tokens a buffer holds */
+    int64_t n_sink;          /* attention-sink prefix that every pruning keeps */
+    int64_t T;               /* in/out: tokens in the cache, <= capacity */
+    uint16_t* const* K[2];   /* HOST arrays of n_layers DEVICE pointers, each bf16 [capacity, n_heads, d_head] */
+    uint16_t* const* V[2];
+    float* SL[2];            /* device fp32 [capacity]: the salience list carried with the cache */
+    int32_t* idx;            /* device int32 [capacity], 16-byte aligned: the index list of the last pruning */
+} pafu_cache;
+
+/* One chunk's update, enqueued on `stream` (nothing is synchronised; the host fields of `cache`
+ * are updated before the call returns and describe the cache once the stream has caught up):
+ *   1. if T + chunk > capacity: idx <- sink prefix + Top-k of SL[0:T] with k such that
+ *      capacity - chunk tokens stay (ties to the lower index, ascending order: pafu_select with
+ *      n_recent = 0); every layer's K and V and SL are gathered through idx into the other buffer
+ *      set (pafu_compact_layers); cur flips; T <- capacity - chunk;
+ *   2. the chunk's scores s = S-MLP([q, k, v]) (pafu_score_qkv on the final layer's rows) are
+ *      written to SL[cur][T : T + chunk];
+ *   3. every layer's new rows are copied to K[cur][l][T : T + chunk], V[cur][l][...]; T += chunk.
+ *   head            as for pafu_score_qkv (d_in = 3 * n_heads * d_head)
+ *   Qs, Ks, Vs      device bf16 [chunk, n_heads, d_head]: the final layer's rows the head reads
+ *   Knew, Vnew      HOST arrays of n_layers DEVICE pointers, each bf16 [chunk, n_heads, d_head]
+ *   pruned          host out, may be NULL: 1 if step 1 ran (cache->idx then holds capacity - chunk indices)
+ *   ws, ws_bytes    as for pafu_score_qkv
+ * Errors (before anything is enqueued): PAFU_ERR_TOO_LARGE if chunk > capacity,
+ * PAFU_ERR_INVALID_ARG for NULL or inconsistent fields (cur not 0/1, T outside [0, capacity], the
+ * two buffer sets sharing a pointer), PAFU_ERR_MISALIGNED, PAFU_ERR_UNSUPPORTED_SHAPE. */
+pafu_status pafu_cache_update(pafu_cache* cache, const pafu_head* head,
+                              const uint16_t* Qs, const uint16_t* Ks, const uint16_t* Vs,
+                              const uint16_t* const* Knew, const uint16_t* const* Vnew, int64_t chunk,
+                              int32_t* pruned, void* ws, size_t ws_bytes, void* stream);
 
 /* Teacher-side salience target - Spatialtemporal-balanced Salience Estimation (Sec. 3.2, Eq. 4
  * and Eq. 5; Algorithm 3).  With P = softmax(scale * Q K^T) per head over the whole sequence of L

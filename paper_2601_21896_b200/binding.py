@@ -29,7 +29,7 @@ STATUS_NAMES = {0: "PAFU_OK", 1: "PAFU_ERR_INVALID_ARG", 2: "PAFU_ERR_BAD_BUDGET
 EXPORTS = ["pafu_version", "pafu_status_string", "pafu_kept_counts", "pafu_workspace_bytes",
            "pafu_workspace_status", "pafu_workspace_counters", "pafu_score", "pafu_score_qkv", "pafu_select", "pafu_compact",
            "pafu_chunk_attn", "pafu_chunk_attn_indexed", "pafu_chunk_attn_noalloc", "pafu_step", "pafu_step_indexed", "pafu_step_timed", "pafu_step_host_arena_bytes", "pafu_step_host", "pafu_step_host_async",
-           "pafu_sse_workspace_bytes", "pafu_sse", "pafu_sse_mean_first", "pafu_compact_layers"]
+           "pafu_sse_workspace_bytes", "pafu_sse", "pafu_sse_mean_first", "pafu_compact_layers", "pafu_cache_update"]
 
 
 class PafuError(RuntimeError):
@@ -59,6 +59,13 @@ class CHead(ctypes.Structure):
 class CPolicy(ctypes.Structure):
     _fields_ = [("n_sink", ctypes.c_int64), ("n_recent", ctypes.c_int64),
                 ("budget", ctypes.c_int64)]
+
+
+class CCache(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("n_heads", ctypes.c_int32), ("d_head", ctypes.c_int32),
+                ("cur", ctypes.c_int32), ("capacity", ctypes.c_int64), ("n_sink", ctypes.c_int64),
+                ("T", ctypes.c_int64), ("K", ctypes.c_void_p * 2), ("V", ctypes.c_void_p * 2),
+                ("SL", ctypes.c_void_p * 2), ("idx", ctypes.c_void_p)]
 
 
 class CStepArgs(ctypes.Structure):
@@ -114,6 +121,9 @@ def lib() -> ctypes.CDLL:
                                               ctypes.c_float, vp, vp, vp, sz, vp]
         L.pafu_step_indexed.restype = i32
         L.pafu_step_indexed.argtypes = [ctypes.POINTER(CStepArgs), vp]
+        L.pafu_cache_update.restype = i32
+        L.pafu_cache_update.argtypes = [ctypes.POINTER(CCache), ctypes.POINTER(CHead), vp, vp, vp, vp, vp, i64,
+                                        ctypes.POINTER(i32), vp, sz, vp]
         L.pafu_compact_layers.restype = i32
         L.pafu_compact_layers.argtypes = [vp, vp, i32, vp, vp, ctypes.POINTER(CShape), ctypes.POINTER(CPolicy),
                                           vp, vp, vp, vp]
@@ -264,6 +274,46 @@ def pafu_compact_layers(Ks, Vs, SL, idx, shape: Shape, policy, Kcs, Vcs, SLc) ->
     arr = lambda ts: (ctypes.c_void_p * max(n, 1))(*[_ptr(t) for t in ts])
     _check(lib().pafu_compact_layers(arr(Ks), arr(Vs), n, _ptr(SL), _ptr(idx), ctypes.byref(shape.c), policy,
                                      arr(Kcs), arr(Vcs), _ptr(SLc), _stream()), "pafu_compact_layers")
+
+
+class Cache:
+    """The rolling KV cache of Algorithm 2 for one stream: two sets of per-layer K / V buffers
+    and salience lists of `capacity` tokens on the current CUDA device, and the host-side counters
+    (`T` tokens in the cache, `cur` the buffer set that holds them)."""
+
+    def __init__(self, n_layers: int, n_heads: int, d_head: int, capacity: int, n_sink: int, device="cuda"):
+        mk = lambda: [torch.zeros((capacity, n_heads, d_head), dtype=torch.bfloat16, device=device) for _ in range(n_layers)]
+        self.Kb, self.Vb = [mk(), mk()], [mk(), mk()]
+        self.SLb = [torch.zeros(capacity, dtype=torch.float32, device=device) for _ in range(2)]
+        self.idx = torch.zeros(capacity, dtype=torch.int32, device=device)
+        arr = lambda ts: (ctypes.c_void_p * n_layers)(*[_ptr(t) for t in ts])
+        self._arrs = [arr(self.Kb[0]), arr(self.Kb[1]), arr(self.Vb[0]), arr(self.Vb[1])]   # kept alive with the struct
+        c = CCache()
+        c.n_layers, c.n_heads, c.d_head, c.cur = n_layers, n_heads, d_head, 0
+        c.capacity, c.n_sink, c.T = capacity, n_sink, 0
+        for b in range(2):
+            c.K[b] = ctypes.cast(self._arrs[b], ctypes.c_void_p)
+            c.V[b] = ctypes.cast(self._arrs[2 + b], ctypes.c_void_p)
+            c.SL[b] = _ptr(self.SLb[b])
+        c.idx = _ptr(self.idx)
+        self.c = c
+
+    T = property(lambda self: int(self.c.T))
+    cur = property(lambda self: int(self.c.cur))
+    K = property(lambda self: [k[: self.T] for k in self.Kb[self.cur]])     # the cache as it stands, per layer
+    V = property(lambda self: [v[: self.T] for v in self.Vb[self.cur]])
+    SL = property(lambda self: self.SLb[self.cur][: self.T])
+
+
+def pafu_cache_update(cache: Cache, head: "Head", Qs, Ks, Vs, Knew, Vnew, ws: torch.Tensor) -> bool:
+    """Algorithm 2's update for one generated chunk; returns True if the cache was pruned first."""
+    n = len(Knew)
+    arr = lambda ts: (ctypes.c_void_p * max(n, 1))(*[_ptr(t) for t in ts])
+    pruned = ctypes.c_int32(0)
+    _check(lib().pafu_cache_update(ctypes.byref(cache.c), ctypes.byref(head.c), _ptr(Qs), _ptr(Ks), _ptr(Vs),
+                                   arr(Knew), arr(Vnew), int(Knew[0].shape[0]) if n else 0, ctypes.byref(pruned),
+                                   _ptr(ws), ws.numel() * ws.element_size(), _stream()), "pafu_cache_update")
+    return bool(pruned.value)
 
 
 def pafu_chunk_attn(Q, Kc, Vc, cu_B, Kq, Vq, shape: Shape, scale: float, O, LSE=None,

@@ -603,4 +603,101 @@ static pafu_status step_host_impl(const pafu_step_args* a, void* arena, size_t a
     return ok ? PAFU_OK : PAFU_ERR_CUDA;
 }
 
+pafu_status pafu_cache_update(pafu_cache* c, const pafu_head* head,
+                              const uint16_t* Qs, const uint16_t* Ks, const uint16_t* Vs,
+                              const uint16_t* const* Knew, const uint16_t* const* Vnew, int64_t chunk,
+                              int32_t* pruned, void* ws, size_t ws_bytes, void* stream) {
+    if (pruned != nullptr) *pruned = 0;
+    if (c == nullptr || chunk < 0) return PAFU_ERR_INVALID_ARG;
+    if (c->n_layers < 1 || c->n_heads < 1 || c->d_head < 1 || c->capacity < 1 || c->n_sink < 0) return PAFU_ERR_INVALID_ARG;
+    if (c->n_layers > PAFU_MAX_LAYERS) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    if (c->cur != 0 && c->cur != 1) return PAFU_ERR_INVALID_ARG;
+    if (c->T < 0 || c->T > c->capacity) return PAFU_ERR_INVALID_ARG;
+    const int64_t dm = (int64_t)c->n_heads * c->d_head;
+    if (dm % 8 != 0 || dm > 0x7fffffffLL || c->capacity > 0x7fffffffLL) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    if (chunk > c->capacity) return PAFU_ERR_TOO_LARGE;
+    if (chunk == 0) return PAFU_OK;
+    pafu_status e = head_ok(head);
+    if (e != PAFU_OK) return e;
+    if (head->d_in != 3 * dm) return PAFU_ERR_INVALID_ARG;
+    if (head->d_in % (64 * 3) != 0) return PAFU_ERR_UNSUPPORTED_SHAPE;
+    if (Qs == nullptr || Ks == nullptr || Vs == nullptr || Knew == nullptr || Vnew == nullptr || c->idx == nullptr)
+        return PAFU_ERR_INVALID_ARG;
+    if (!aligned16(Qs) || !aligned16(Ks) || !aligned16(Vs) || !aligned16(c->idx)) return PAFU_ERR_MISALIGNED;
+    const size_t buf_b = (size_t)c->capacity * dm * 2;
+    for (int b = 0; b < 2; ++b) {
+        if (c->K[b] == nullptr || c->V[b] == nullptr || c->SL[b] == nullptr) return PAFU_ERR_INVALID_ARG;
+        if (!aligned16(c->SL[b])) return PAFU_ERR_MISALIGNED;
+    }
+    if (ranges_overlap(c->SL[0], (size_t)c->capacity * 4, c->SL[1], (size_t)c->capacity * 4)) return PAFU_ERR_INVALID_ARG;
+    for (int l = 0; l < c->n_layers; ++l) {
+        if (Knew[l] == nullptr || Vnew[l] == nullptr) return PAFU_ERR_INVALID_ARG;
+        if (!aligned16(Knew[l]) || !aligned16(Vnew[l])) return PAFU_ERR_MISALIGNED;
+        const void* bufs[4] = {c->K[0][l], c->V[0][l], c->K[1][l], c->V[1][l]};
+        for (int i = 0; i < 4; ++i) {
+            if (bufs[i] == nullptr) return PAFU_ERR_INVALID_ARG;
+            if (!aligned16(bufs[i])) return PAFU_ERR_MISALIGNED;
+            // a layer's four buffers are distinct, and none of them is where the new rows come from
+            for (int j = i + 1; j < 4; ++j)
+                if (ranges_overlap(bufs[i], buf_b, bufs[j], buf_b)) return PAFU_ERR_INVALID_ARG;
+            if (ranges_overlap(bufs[i], buf_b, Knew[l], (size_t)chunk * dm * 2) ||
+                ranges_overlap(bufs[i], buf_b, Vnew[l], (size_t)chunk * dm * 2)) return PAFU_ERR_INVALID_ARG;
+        }
+    }
+    if (ws == nullptr) return PAFU_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PAFU_ERR_MISALIGNED;
+    if (ws_bytes < kWsHeaderBytes + score_workspace_bytes(*head)) return PAFU_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+    // 1. the chunk does not fit: keep the sink prefix and the Top-k of SL, in every layer
+    if (c->T + chunk > c->capacity) {
+        const int64_t keep = c->capacity - chunk;
+        if (keep > 0) {
+            StreamTable st;
+            memset(&st, 0, sizeof st);
+            st.n_streams = 1;
+            st.cu_T[1] = c->T;
+            pafu_shape sh;
+            memset(&sh, 0, sizeof sh);
+            sh.n_streams = 1; sh.n_heads = c->n_heads; sh.d_head = c->d_head; sh.cu_T = st.cu_T;
+            pafu_policy pol;
+            pol.n_sink = c->n_sink; pol.n_recent = 0; pol.budget = keep;
+            e = fill_policy(&sh, &pol, &st);
+            if (e != PAFU_OK) return e;
+            e = launch_select(c->SL[c->cur], st, c->idx, cs);
+            if (e != PAFU_OK) return e;
+            const int o = c->cur ^ 1;
+            e = launch_compact_layers(c->K[c->cur], c->V[c->cur], c->n_layers, c->SL[c->cur], c->idx, st, (int32_t)dm,
+                                      c->K[o], c->V[o], c->SL[o], cs);
+            if (e != PAFU_OK) return e;
+        }
+        c->cur ^= 1;
+        c->T = keep;
+        if (pruned != nullptr) *pruned = 1;
+    }
+    // 2. the chunk's salience scores go straight to the tail of SL
+    const uint16_t* parts[3] = {Qs, Ks, Vs};
+    e = launch_score(*head, parts, 3, chunk, dm, c->SL[c->cur] + c->T, ws, ws_bytes, cs);
+    if (e != PAFU_OK) return e;
+    // 3. every layer's new rows go to the tail of its K and V
+    {
+        StreamTable st;
+        memset(&st, 0, sizeof st);
+        st.n_streams = 1;
+        st.cu_T[1] = chunk;
+        st.cu_B[1] = chunk;
+        const uint16_t* kd[PAFU_MAX_LAYERS]; const uint16_t* vd[PAFU_MAX_LAYERS];
+        uint16_t* ko[PAFU_MAX_LAYERS]; uint16_t* vo[PAFU_MAX_LAYERS];
+        for (int l = 0; l < c->n_layers; ++l) {
+            kd[l] = Knew[l]; vd[l] = Vnew[l];
+            ko[l] = c->K[c->cur][l] + c->T * dm;
+            vo[l] = c->V[c->cur][l] + c->T * dm;
+        }
+        e = launch_compact_layers(kd, vd, c->n_layers, nullptr, nullptr, st, (int32_t)dm, ko, vo, nullptr, cs);
+        if (e != PAFU_OK) return e;
+    }
+    c->T += chunk;
+    return PAFU_OK;
+}
+
 }  // extern "C"

@@ -179,7 +179,8 @@ compact_layers_kernel(const __grid_constant__ LayerPtrs lp, int32_t n_layers,
         const int64_t r = w - (int64_t)layer * n_rows;
         int s = 0;
         while (s + 1 < st.n_streams && r >= st.cu_B[s + 1]) ++s;
-        const int64_t src_row = st.cu_T[s] + (int64_t)__ldg(idx + r);
+        // idx == nullptr: the rows in order (a plain copy of every layer's rows)
+        const int64_t src_row = st.cu_T[s] + (idx != nullptr ? (int64_t)__ldg(idx + r) : r - st.cu_B[s]);
         const uint4* ks = lp.K[layer] + src_row * chunks_per_row;
         const uint4* vs = lp.V[layer] + src_row * chunks_per_row;
         uint4* kd = lp.Kc[layer] + r * chunks_per_row;

@@ -42,6 +42,7 @@ def test_struct_layouts_match_header():
     assert ctypes.sizeof(B.CHead) == 56
     assert ctypes.sizeof(B.CPolicy) == 24
     assert ctypes.sizeof(B.CStepArgs) == 32 + 8 + 8 + 5 * 8 + 8 + 7 * 8 + 8 + 8
+    assert ctypes.sizeof(B.CCache) == 4 * 4 + 3 * 8 + 6 * 8 + 8
 
 
 def test_kept_counts_and_clamping(L):
@@ -170,6 +171,50 @@ def test_overlap_and_host_step_checks_run_before_anything_is_enqueued(L):
     assert L.pafu_step_host(ctypes.byref(args(head(256, 32, 0))), arena + 8, big, None) == 5  # arena alignment
     assert L.pafu_step_host(ctypes.byref(args(head(256, 32, 0))), arena, 1024, None) == 4     # arena too small
     assert L.pafu_workspace_counters(None, None, None) == 1
+
+
+def test_cache_update_rejects_bad_arguments_on_host(L):
+    """Every refusal of pafu_cache_update comes before anything is enqueued and leaves the
+    host counters as they were (fake device addresses: nothing may be touched)."""
+    fake = 0x7f0000000000
+    n_layers, N, D, cap, chunk = 2, 2, 64, 1024, 256
+    dm, MB = N * D, 1 << 20
+    def make(cur=0, T=0, capacity=cap, share=False, sl_same=False):
+        ptrs = lambda base: (ctypes.c_void_p * n_layers)(*[base + l * MB for l in range(n_layers)])
+        arrs = [ptrs(fake + 16 * MB), ptrs(fake + (16 if share else 32) * MB), ptrs(fake + 48 * MB), ptrs(fake + 64 * MB)]
+        c = B.CCache()
+        c.n_layers, c.n_heads, c.d_head, c.cur, c.capacity, c.n_sink, c.T = n_layers, N, D, cur, capacity, 16, T
+        c.K[0], c.K[1] = ctypes.cast(arrs[0], ctypes.c_void_p), ctypes.cast(arrs[1], ctypes.c_void_p)
+        c.V[0], c.V[1] = ctypes.cast(arrs[2], ctypes.c_void_p), ctypes.cast(arrs[3], ctypes.c_void_p)
+        c.SL[0], c.SL[1] = fake + 96 * MB, fake + (96 if sl_same else 97) * MB
+        c.idx = fake + 98 * MB
+        return c, arrs
+    head = B.CHead(3 * dm, 64, 12, 1, 0, fake + 100 * MB, None, fake + 101 * MB, None)
+    new = (ctypes.c_void_p * n_layers)(fake + 110 * MB, fake + 111 * MB)
+    def call(c, ch=chunk, hd=head, kn=new, ws=fake + 120 * MB, nb=1 << 20):
+        pr = ctypes.c_int32(7)
+        rc = L.pafu_cache_update(ctypes.byref(c), ctypes.byref(hd) if hd is not None else None, fake, fake, fake, kn, new, ch,
+                                 ctypes.byref(pr), ws, nb, None)
+        return rc, pr.value
+    c, keep = make(T=300)
+    assert call(c, ch=cap + 1) == (8, 0) and (c.T, c.cur) == (300, 0)          # chunk longer than the cache
+    assert call(c, ch=-1)[0] == 1
+    assert call(c, ch=0) == (0, 0) and c.T == 300                               # nothing to append: no-op
+    assert call(make(cur=2)[0])[0] == 1
+    assert call(make(T=cap + 1)[0])[0] == 1
+    assert call(make(share=True)[0])[0] == 1                                    # the two buffer sets share storage
+    assert call(make(sl_same=True)[0])[0] == 1
+    assert call(c, hd=None)[0] == 1
+    assert call(c, hd=B.CHead(2 * dm, 64, 12, 1, 0, fake, None, fake, None))[0] == 1   # head does not read [q, k, v]
+    assert call(c, kn=(ctypes.c_void_p * n_layers)(fake + 110 * MB, None))[0] == 1
+    assert call(c, kn=(ctypes.c_void_p * n_layers)(fake + 110 * MB, fake + 111 * MB + 2))[0] == 5
+    assert call(c, kn=(ctypes.c_void_p * n_layers)(fake + 16 * MB, fake + 111 * MB))[0] == 1   # new rows inside a cache buffer
+    assert call(c, ws=None)[0] == 1
+    assert call(c, ws=fake + 120 * MB + 64)[0] == 5
+    assert call(c, nb=16)[0] == 4
+    c65, _ = make(); c65.n_layers = 65
+    assert call(c65)[0] == 3
+    assert (c.T, c.cur) == (300, 0)
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

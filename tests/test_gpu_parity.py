@@ -448,6 +448,51 @@ def test_algorithm2_cache_update_over_chunks():
         assert np.array_equal(K[l][:n_sink], first_K[l][:n_sink])
 
 
+@pytest.mark.parametrize("chunk,cap,n_sink", [(96, 320, 32), (101, 323, 17), (64, 64, 8)])
+def test_cache_update_entry_point_over_chunks(chunk, cap, n_sink):
+    """pafu_cache_update (Algorithm 2's whole per-chunk update in one call: prune every layer with
+    one index list when the chunk does not fit, score the chunk into the tail of SL, append the
+    chunk's rows) against oracle.cache_update, chunk after chunk: caches, SL and the index list
+    bit-identical (the mirror appends the GPU's own fp32 scores), the scores within tolerance of
+    the oracle's S-MLP.  Sizes with a ragged tail, an SL tail that is not 16-byte aligned, and a
+    cache that holds exactly one chunk (every update replaces everything)."""
+    rng = np.random.default_rng(41)
+    N, D, n_layers = 2, 128, 3
+    dm = N * D
+    bits = lambda shape, sc=1.0: wl.f32_to_bf16_bits((rng.standard_normal(shape) * sc).astype(np.float32))
+    w1, b1 = bits((64, 3 * dm), (3 * dm) ** -0.5), bits((64,), 0.3)
+    w2, b2 = bits((12, 64), 64 ** -0.5), bits((12,), 0.3)
+    dw = [to_device_bf16(a) for a in (w1, b1, w2, b2)]
+    head = pafu.Head(dw[0], dw[1], dw[2], dw[3], wl.ACT_SILU, wl.FINAL_NONE)
+    ws = torch.zeros(pafu.pafu_workspace_bytes(pafu.Shape(N, D, [0, cap], [0, chunk]), None, head),
+                     dtype=torch.uint8, device="cuda")
+    cache = pafu.Cache(n_layers, N, D, cap, n_sink)
+    K = [np.zeros((0, N, D), np.uint16) for _ in range(n_layers)]; V = [k.copy() for k in K]     # mirror
+    SL = np.zeros(0, np.float32)
+    n_pruned = 0
+    for c in range(7):
+        newK = [bits((chunk, N, D)) for _ in range(n_layers)]; newV = [bits((chunk, N, D)) for _ in range(n_layers)]
+        q = bits((chunk, N, D))
+        T_before, cur_before = cache.T, cache.cur
+        pruned = pafu.pafu_cache_update(cache, head, to_device_bf16(q), to_device_bf16(newK[-1]), to_device_bf16(newV[-1]),
+                                        [to_device_bf16(a) for a in newK], [to_device_bf16(a) for a in newV], ws)
+        assert pruned == (T_before + chunk > cap) and cache.cur == (cur_before ^ int(pruned))
+        n_pruned += int(pruned)
+        assert pafu.pafu_workspace_status(ws) == 0
+        s_gpu = cache.SL[cache.T - chunk:].cpu().numpy()
+        X = np.concatenate([q.reshape(chunk, dm), newK[-1].reshape(chunk, dm), newV[-1].reshape(chunk, dm)], axis=1)
+        close(s_gpu, oracle.score(np.ascontiguousarray(X), w1, b1, w2, b2, wl.ACT_SILU, wl.FINAL_NONE), "chunk score")
+        K, V, SL, ids = oracle.cache_update(K, V, SL, newK, newV, s_gpu, cap, n_sink)
+        assert (ids is not None) == pruned
+        if pruned:
+            assert np.array_equal(cache.idx[: cap - chunk].cpu().numpy(), ids)
+        assert cache.T == SL.shape[0] <= cap
+        assert np.array_equal(cache.SL.cpu().numpy(), SL)
+        for l in range(n_layers):
+            assert np.array_equal(bf16_to_bits(cache.K[l]), K[l]) and np.array_equal(bf16_to_bits(cache.V[l]), V[l]), (c, l)
+    assert n_pruned >= 3
+
+
 # --------------------------------------------------------------- attention through indices
 def test_indexed_attention_matches_oracle_and_compacted_path():
     """Select(KV; ids) applied inside the attention loader (Eq. 7's index set) instead of as a
