@@ -638,6 +638,37 @@ def run_ours(args):
                   "GB/s": c_bytes / (c_ms * 1e-3) / 1e9, "hbm_frac": c_bytes / (c_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         del Ks, Vs, Kcs, Vcs
 
+    # ---- Algorithm 2's per-chunk cache update as one call, at the paper's own operating point
+    # (Sec. 3.4 / Appendix A: a cache of 9360 tokens pruned to 4680 when the next 4680-token chunk
+    # arrives), all 30 layers, steady state: every update prunes, scores the chunk with the paper's
+    # S-MLP and appends.  3.45 GB of K/V rows move per update, far more than L2 holds.
+    cache_upd = None
+    if rank == 0 and qkv is not None and args.shared_layers == N_LAYERS_PER_DENOISE_STEP and w.d_head == 128:
+        nl, cap, ch = N_LAYERS_PER_DENOISE_STEP, 2 * wl.CHUNK_TOKENS, wl.CHUNK_TOKENS
+        cache = pafu.Cache(nl, w.n_heads, w.d_head, cap, wl.TOKENS_PER_FRAME)
+        g = torch.Generator(device="cuda"); g.manual_seed(3)
+        newK = [torch.randn((ch, w.n_heads, w.d_head), generator=g, device="cuda").to(torch.bfloat16) for _ in range(nl)]
+        newV = [torch.randn((ch, w.n_heads, w.d_head), generator=g, device="cuda").to(torch.bfloat16) for _ in range(nl)]
+        qn = torch.randn((ch, w.n_heads, w.d_head), generator=g, device="cuda").to(torch.bfloat16)
+        ev_u = [new_events(2) for _ in range(6)]
+        n_pruned = 0
+        for r in range(9):
+            if r >= 3:
+                ev_u[r - 3][0].record(stream)
+            pr = pafu.pafu_cache_update(cache, phead, qn, newK[-1], newV[-1], newK, newV, pws)
+            if r >= 3:
+                ev_u[r - 3][1].record(stream)
+                n_pruned += int(pr)
+        torch.cuda.synchronize()
+        assert pafu.pafu_workspace_status(pws) == 0 and n_pruned == 6 and cache.T == cap
+        u_ms = float(np.median([a.elapsed_time(b) for a, b in ev_u]))
+        row_b = w.d_model * 2
+        u_bytes = nl * 2 * 2 * (cap - ch) * row_b + nl * 2 * 2 * ch * row_b + ch * 3 * row_b
+        cache_upd = {"workload": "pafu_cache_update, %d layers, cache %d -> %d + chunk %d, paper S-MLP" % (nl, cap, cap - ch, ch),
+                     "ms": u_ms, "GB/s": u_bytes / (u_ms * 1e-3) / 1e9,
+                     "hbm_frac": u_bytes / (u_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "launches": 4}
+        del cache, newK, newV
+
     # ---- teacher salience target (Eq. 4, Eq. 5) at the paper's training length: 21 frames of
     # 1560 tokens, blocks of 4680 (Appendix A).  200 MB of Q and K: larger than L2.
     sse = None
@@ -721,6 +752,7 @@ def run_ours(args):
         "cuda_graph": graph,
         "sse": sse,
         "shared_index_compaction": shared,
+        "cache_update": cache_upd,
         "layers_per_step": n_layers,
         "ms_per_denoise_step_30_layers": N_LAYERS_PER_DENOISE_STEP * ms_per_step / n_layers,
         # the paper's own schedule (Sec. 3.3, Algorithm 2): score the new chunk and prune every layer's
@@ -728,8 +760,10 @@ def run_ours(args):
         "paper_schedule": None if not (qkv and shared and args.shared_layers == N_LAYERS_PER_DENOISE_STEP) else {
             "prune_once_per_chunk_ms": qkv["ms"] + shared["ms"],
             "attention_per_denoise_step_30_layers_ms": N_LAYERS_PER_DENOISE_STEP * k["attn"]["median"] * 1e-3,
-            "note": "S-MLP on the chunk's [q,k,v] + one select + 30-layer shared-index compaction; "
-                    "30 x (attention + merge) per denoising step"},
+            "cache_update_ms_at_9360_to_4680": None if cache_upd is None else cache_upd["ms"],
+            "note": "S-MLP on the chunk's [q,k,v] + one select + 30-layer shared-index compaction at this "
+                    "workload's cache size; cache_update: the same plus the append, one call, at the paper's "
+                    "own cache size; 30 x (attention + merge) per denoising step"},
         "configs": configs,
         "peaks": dict(peaks, nominal=NOMINAL),
         "clocks": clocks,
