@@ -9,18 +9,18 @@
 namespace pafu {
 
 size_t attn_workspace_bytes(const StreamTable&, int32_t, int32_t d_head) {
-    return d_head == attn_tc::kD ? attn_tc::workspace_bytes() : 0;
+    return (d_head == attn_tc::kD || d_head == 64) ? attn_tc::workspace_bytes() : 0;
 }
 
 pafu_status launch_attn(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
                         const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
                         int32_t n_heads, int32_t d_head, float scale, uint16_t* O, float* LSE,
                         void* ws, size_t, cudaStream_t stream) {
-    if (d_head == attn_tc::kD && attn_tc::supports(st, Kq != nullptr)) {
+    if ((d_head == attn_tc::kD || d_head == 64) && attn_tc::supports(st, Kq != nullptr)) {
         uint8_t* base = static_cast<uint8_t*>(ws);
         return attn_tc::launch(Q, Kc, Vc, Kq, Vq, st, n_heads, scale, O, LSE,
                                reinterpret_cast<int*>(base) + kStatusWordTimeout,
-                               reinterpret_cast<float*>(base + kWsHeaderBytes), stream);
+                               reinterpret_cast<float*>(base + kWsHeaderBytes), stream, 0, nullptr, d_head);
     }
     return attn_mma::launch(Q, Kc, Vc, Kq, Vq, st, n_heads, d_head, scale, O, LSE, stream);
 }
@@ -33,8 +33,7 @@ pafu_status launch_attn_indexed(const uint16_t* Q, const uint16_t* K, const uint
     uint8_t* base = static_cast<uint8_t*>(ws);
     return attn_tc::launch(Q, K, V, Kq, Vq, st, n_heads, scale, O, LSE,
                            reinterpret_cast<int*>(base) + kStatusWordTimeout,
-                           reinterpret_cast<float*>(base + kWsHeaderBytes), stream, 0, idx,
-                           st.cu_T[st.n_streams]);
+                           reinterpret_cast<float*>(base + kWsHeaderBytes), stream, 0, idx);
 }
 
 bool attn_indexed_supported(const StreamTable& st, int32_t d_head, bool has_chunk) {

@@ -3,8 +3,8 @@
 // o_i = sum_j softmax_j(scale q_i.k_j) v_j with j over [retained cache ; chunk tokens]
 // (Sec. 3.2 for the operator; Eq. 2 / Eq. 7 for the key range).  One CTA of 4 warps owns 64
 // query rows of one head and streams 64-key tiles of both key segments through shared memory
-// with an online softmax.  It serves the shapes the tcgen05 kernel does not take (d_head 64,
-// short inputs) and is the kernel of record for them.
+// with an online softmax.  It serves the inputs the tcgen05 kernel does not take: a stream that
+// has queries but not a single key (no retained cache and no chunk segment), whose rows are zero.
 #pragma once
 #include "common.cuh"
 

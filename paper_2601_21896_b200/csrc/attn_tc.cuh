@@ -1,4 +1,5 @@
-// Chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), d_head = 128.
+// Chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), d_head = 128 (and 64:
+// a second instantiation, see HeadDims; the text below gives the sizes for 128).
 //
 //   o_i = sum_j softmax_j(scale q_i.k_j) v_j,  j over [retained cache ; chunk tokens]
 //   (Sec. 3.2 for the operator; Eq. 2 / Eq. 7 for the key range)
@@ -203,11 +204,29 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // maps of it).  GATHER = true: they are rows idx[.] of the uncompacted cache, fetched by the
 // loader warp with 16-byte asynchronous copies (mKc, mVc unused); everything downstream of the
 // shared-memory ring is identical.
-template <bool GATHER>
+// Sizes that depend on the head width D (128, or 64: every tile is then a single 64-column
+// swizzled block, S = Q K^T takes four slices and O has 64 columns).
+template <int D>
+struct HeadDims {
+    static constexpr int kQBytes = kBM * D * 2;                  // one slot's Q tile
+    static constexpr int kQHalf = kBM * 64 * 2;                  // one [128 rows x 64 cols] swizzled block of it
+    static constexpr int kHalfBytes = kBN * 64 * 2;              // one [64 rows x 64 cols] swizzled block of a K or V tile
+    static constexpr int kTileBytes = kBN * D * 2;
+    static constexpr int kSmemBytes = 2 * kQBytes + kStages * kTileBytes + 1024 /*align*/ + 512 /*barriers*/;
+    static constexpr int kPieceFloats = 2 * kBM * D + 2 * 2 * kBM;   // one partial: O [256][D], m [256], l [256]
+};
+
+template <bool GATHER, int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mKc,
                const __grid_constant__ CUtensorMap mVc, const __grid_constant__ CUtensorMap mKq,
                const __grid_constant__ CUtensorMap mVq, const __grid_constant__ Params p) {
+    static_assert(D == 128 || (D == 64 && !GATHER), "head widths: 128, or 64 with a compacted cache");
+    // this instantiation's sizes (they shadow the D = 128 constants of the namespace)
+    constexpr int kD = D;
+    constexpr int kQBytes = HeadDims<D>::kQBytes, kQHalf = HeadDims<D>::kQHalf;
+    constexpr int kTileBytes = HeadDims<D>::kTileBytes, kHalfBytes = HeadDims<D>::kHalfBytes;
+    constexpr int kPieceFloats = HeadDims<D>::kPieceFloats;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sQ = smem_u32(smem);                       // 2 slots x 32 KiB
@@ -302,7 +321,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                         if (lane == 0) {
                             mbar_arrive_expect_tx(q_full(s), kQBytes);
                             tma_load_3d(sQ + s * kQBytes, &mQ, q_full(s), 0, g.head, qrow + s * kBM);
-                            tma_load_3d(sQ + s * kQBytes + kQHalf, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
+                            if constexpr (D == 128) tma_load_3d(sQ + s * kQBytes + kQHalf, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
                         }
                     }
                 }
@@ -335,7 +354,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                             const int row2 = (int)(p.st.cu_Lq[g.stream] + (int64_t)(j - g.nt1) * kBN);
                             mbar_arrive_expect_tx(kv_full(st), kTileBytes);
                             tma_load_3d(sKV + st * kTileBytes, m, kv_full(st), 0, g.head, row2);
-                            tma_load_3d(sKV + st * kTileBytes + kHalfBytes, m, kv_full(st), 64, g.head, row2);
+                            if constexpr (D == 128) tma_load_3d(sKV + st * kTileBytes + kHalfBytes, m, kv_full(st), 64, g.head, row2);
                         } else {
                             mbar_arrive(kv_full(st));
                         }
@@ -372,7 +391,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                     if (s) ++qcnt1; else ++qcnt0;
                     mbar_arrive_expect_tx(q_full(s), kQBytes);
                     tma_load_3d(sQ + s * kQBytes, &mQ, q_full(s), 0, g.head, qrow + s * kBM);
-                    tma_load_3d(sQ + s * kQBytes + kQHalf, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
+                    if constexpr (D == 128) tma_load_3d(sQ + s * kQBytes + kQHalf, &mQ, q_full(s), 64, g.head, qrow + s * kBM);
                 }
                 for (int j = g.t0; j < g.t1 && ok; ++j) {
                     const bool seg2 = j >= g.nt1;
@@ -385,7 +404,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                         const CUtensorMap* m = seg2 ? (kv ? &mVq : &mKq) : (kv ? &mVc : &mKc);
                         mbar_arrive_expect_tx(kv_full(st), kTileBytes);
                         tma_load_3d(sKV + st * kTileBytes, m, kv_full(st), 0, g.head, row);
-                        tma_load_3d(sKV + st * kTileBytes + kHalfBytes, m, kv_full(st), 64, g.head, row);
+                        if constexpr (D == 128) tma_load_3d(sKV + st * kTileBytes + kHalfBytes, m, kv_full(st), 64, g.head, row);
                     }
                 }
             }
@@ -598,7 +617,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                         l_sum *= alpha;
                         m_used = m_new;
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
+                        for (int c = 0; c < kD / 32; ++c) {
                             uint32_t orr[32];
                             PAFU_TMEM_LD_X32(tO + c * 32, orr);
                             tmem_wait_ld();
@@ -653,7 +672,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 const float inv = (l_sum > 0.f) ? 1.0f / l_sum : 0.f;
                 uint16_t* dst = p.O + ((p.st.cu_Lq[g.stream] + row) * p.n_heads + g.head) * kD;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < kD / 32; ++c) {
                     uint32_t orr[32];
                     PAFU_TMEM_LD_X32(tO + c * 32, orr);
                     tmem_wait_ld();
@@ -678,7 +697,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ C
                 const int prow = slot * kBM + row_in_slot;
                 float4* dst = reinterpret_cast<float4*>(piece + (size_t)prow * kD);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < kD / 32; ++c) {
                     uint32_t orr[32];
                     PAFU_TMEM_LD_X32(tO + c * 32, orr);
                     tmem_wait_ld();
@@ -718,9 +737,12 @@ struct MergeTable {
     int16_t cta[2 * kMaxGrid];
 };
 
+template <int D>
 __global__ void __launch_bounds__(kMergeThreads)
 attn_tc_merge_kernel(const __grid_constant__ MergeTable tb, const float* __restrict__ pieces, float scale,
                      int n_heads, int64_t total_Lq, uint16_t* __restrict__ O, float* __restrict__ LSE) {
+    constexpr int kD = D;
+    constexpr int kPieceFloats = HeadDims<D>::kPieceFloats;
     grid_dep_wait();
     const MergeItem& it = tb.item[blockIdx.x / kMergeBlocksPerItem];
     const int slot = (blockIdx.x / (kMergeBlocksPerItem / 2)) & 1;
@@ -748,7 +770,7 @@ attn_tc_merge_kernel(const __grid_constant__ MergeTable tb, const float* __restr
             const int r = slot * kBM + r0 + q;
             w[q] = piece[2 * kBM * kD + r];
             l[q] = piece[2 * kBM * kD + 2 * kBM + r];
-            v[q] = reinterpret_cast<const float4*>(piece + (size_t)r * kD)[lane];
+            v[q] = lane < kD / 4 ? reinterpret_cast<const float4*>(piece + (size_t)r * kD)[lane] : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
         for (int q = 0; q < kMergeRows; ++q) {
@@ -766,7 +788,7 @@ attn_tc_merge_kernel(const __grid_constant__ MergeTable tb, const float* __restr
         uint2 o;
         o.x = pack_bf16(acc[q].x * inv, acc[q].y * inv);
         o.y = pack_bf16(acc[q].z * inv, acc[q].w * inv);
-        *reinterpret_cast<uint2*>(dst) = o;
+        if (lane < kD / 4) *reinterpret_cast<uint2*>(dst) = o;
         if (LSE != nullptr && lane == 0)
             LSE[(int64_t)it.head * total_Lq + it.o_row + row] = (L[q] > 0.f) ? M[q] * scale + logf(L[q]) : -INFINITY;
     }
@@ -824,54 +846,72 @@ inline bool supports(const StreamTable& st, bool has_chunk) {
 inline size_t workspace_bytes() { return (size_t)sm_count() * 2 * kPieceBytes; }
 
 // Tensor maps are rebuilt per call (a few microseconds of host work); nothing is cached, so
-// the library stays stateless.
-inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
-                          const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
-                          int32_t n_heads, float scale, uint16_t* O, float* LSE, int* status,
-                          float* pieces, cudaStream_t stream, int max_ctas = 0,
-                          const int32_t* idx = nullptr, int64_t n_cache_rows = 0) {
+// the library stays stateless.  D: head width (128; 64 with a compacted cache only).
+template <int D>
+inline pafu_status launch_d(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
+                            const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
+                            int32_t n_heads, float scale, uint16_t* O, float* LSE, int* status,
+                            float* pieces, cudaStream_t stream, int max_ctas, const int32_t* idx) {
+    constexpr int kSmem = HeadDims<D>::kSmemBytes;
     const int n = st.n_streams;
     const int64_t nQ = st.cu_Lq[n], nB = st.cu_B[n];
     const int has_chunk = Kq != nullptr;
     const int64_t cost = total_cost(st, n_heads, has_chunk);
     if (cost == 0) return PAFU_OK;
     CUtensorMap mQ, mKc, mVc, mKq, mVq;
-    if (!TmapEncoder::token_tensor(&mQ, Q, (uint64_t)nQ, n_heads, kD, kBM)) return PAFU_ERR_CUDA;
-    const bool gather = idx != nullptr;      // Kc, Vc are then the uncompacted cache of n_cache_rows tokens
+    if (!TmapEncoder::token_tensor(&mQ, Q, (uint64_t)nQ, n_heads, D, kBM)) return PAFU_ERR_CUDA;
+    const bool gather = idx != nullptr;      // Kc, Vc are then the uncompacted cache
+    if (gather && D != 128) return PAFU_ERR_UNSUPPORTED_SHAPE;
     if (nB > 0 && gather) {
         mKc = mQ; mVc = mQ;                 // the gather loader reads the cache through plain pointers
-        (void)n_cache_rows;
     } else if (nB > 0) {
-        if (!TmapEncoder::token_tensor(&mKc, Kc, (uint64_t)nB, n_heads, kD, kBN) ||
-            !TmapEncoder::token_tensor(&mVc, Vc, (uint64_t)nB, n_heads, kD, kBN)) return PAFU_ERR_CUDA;
+        if (!TmapEncoder::token_tensor(&mKc, Kc, (uint64_t)nB, n_heads, D, kBN) ||
+            !TmapEncoder::token_tensor(&mVc, Vc, (uint64_t)nB, n_heads, D, kBN)) return PAFU_ERR_CUDA;
     } else { mKc = mQ; mVc = mQ; }
     if (has_chunk) {
-        if (!TmapEncoder::token_tensor(&mKq, Kq, (uint64_t)nQ, n_heads, kD, kBN) ||
-            !TmapEncoder::token_tensor(&mVq, Vq, (uint64_t)nQ, n_heads, kD, kBN)) return PAFU_ERR_CUDA;
+        if (!TmapEncoder::token_tensor(&mKq, Kq, (uint64_t)nQ, n_heads, D, kBN) ||
+            !TmapEncoder::token_tensor(&mVq, Vq, (uint64_t)nQ, n_heads, D, kBN)) return PAFU_ERR_CUDA;
     } else { mKq = mQ; mVq = mQ; }
     Params p;
     p.st = st; p.n_heads = n_heads; p.has_chunk = has_chunk; p.scale = scale;
     p.O = O; p.LSE = LSE; p.status = status; p.pieces = pieces; p.idx = idx; p.Kraw = gather ? Kc : nullptr; p.Vraw = gather ? Vc : nullptr; p.total_Lq = nQ; p.total_cost = cost;
     static bool attr_set[kMaxDevices] = {};
     if (!once_per_device(attr_set, [] {
-            return cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess &&
-                   cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) == cudaSuccess;
+            if (cudaFuncSetAttribute(attn_tc_kernel<false, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) return false;
+            if constexpr (D == 128)
+                return cudaFuncSetAttribute(attn_tc_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) == cudaSuccess;
+            return true;
         }))
         return PAFU_ERR_CUDA;
     int grid = grid_for(cost);
     if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;   // caller's scratch holds fewer partials
-    if ((gather ? launch_dependent(attn_tc_kernel<true>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mKc, mVc, mKq, mVq, p)
-                : launch_dependent(attn_tc_kernel<false>, dim3(grid), dim3(kThreads), kSmemBytes, stream, 1, mQ, mKc, mVc, mKq, mVq, p)) != cudaSuccess)
-        return PAFU_ERR_CUDA;
+    cudaError_t le;
+    if constexpr (D == 128) {
+        le = gather ? launch_dependent(attn_tc_kernel<true, 128>, dim3(grid), dim3(kThreads), kSmem, stream, 1, mQ, mKc, mVc, mKq, mVq, p)
+                    : launch_dependent(attn_tc_kernel<false, 128>, dim3(grid), dim3(kThreads), kSmem, stream, 1, mQ, mKc, mVc, mKq, mVq, p);
+    } else {
+        le = launch_dependent(attn_tc_kernel<false, D>, dim3(grid), dim3(kThreads), kSmem, stream, 1, mQ, mKc, mVc, mKq, mVq, p);
+    }
+    if (le != cudaSuccess) return PAFU_ERR_CUDA;
     if (grid > 1) {
         MergeTable tb;
         build_merge_table(p, grid, tb);
         if (tb.n_items > 0 &&
-            launch_dependent(attn_tc_merge_kernel, dim3(tb.n_items * kMergeBlocksPerItem), dim3(kMergeThreads), 0, stream, 1,
+            launch_dependent(attn_tc_merge_kernel<D>, dim3(tb.n_items * kMergeBlocksPerItem), dim3(kMergeThreads), 0, stream, 1,
                              tb, (const float*)pieces, scale, (int)n_heads, nQ, O, LSE) != cudaSuccess)
             return PAFU_ERR_CUDA;
     }
     return PAFU_OK;
+}
+
+inline pafu_status launch(const uint16_t* Q, const uint16_t* Kc, const uint16_t* Vc,
+                          const uint16_t* Kq, const uint16_t* Vq, const StreamTable& st,
+                          int32_t n_heads, float scale, uint16_t* O, float* LSE, int* status,
+                          float* pieces, cudaStream_t stream, int max_ctas = 0,
+                          const int32_t* idx = nullptr, int d_head = kD) {
+    if (d_head == 64)
+        return launch_d<64>(Q, Kc, Vc, Kq, Vq, st, n_heads, scale, O, LSE, status, pieces, stream, max_ctas, idx);
+    return launch_d<128>(Q, Kc, Vc, Kq, Vq, st, n_heads, scale, O, LSE, status, pieces, stream, max_ctas, idx);
 }
 
 }  // namespace attn_tc
